@@ -1,0 +1,273 @@
+/*
+ * CPU oracle for the Hyper-Parallel Decoding (HPD) decode step.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition that the CUDA
+ * path is checked against.  It shares no code, header, table or helper with the CUDA
+ * library and must never be called from the product path; only the test-suite, the
+ * smoke check and the benchmark's cpu-baseline leg execute it.
+ *
+ * What it computes (each function cites the passage it follows):
+ *   - position IDs with K_max gaps                      Algorithm 2, Sec. 4.3.1
+ *   - per-step bookkeeping tables for live branches      Sec. 4.3.2-4.3.6 (append order,
+ *                                                        IDs = previous + 1, pruning, b*J*N rows)
+ *   - rotary embedding at an assigned position ID        Sec. 4.3.1 ("position IDs define
+ *                                                        positional embeddings"), Sec. 4.4
+ *   - per-branch attention                               Eq. 5-6: a value token depends on the
+ *                                                        prompt and on its own earlier tokens only
+ *
+ * Precision: inputs are fp32 values (the harness widens bf16 exactly); every product,
+ * sum, exponential and trigonometric value is taken in fp64.  There is no blocking,
+ * no online softmax, no fusion: the concatenated sequence of a branch is materialised
+ * and ordinary causal attention is evaluated on it.
+ *
+ * Parity pins (tests marked "not gpu"): Algorithm 2 against the position numbers the
+ * paper prints for its K_max = 7 figure; rope against closed forms and the relative-
+ * position identity; attention against a full-matrix masked softmax in numpy, against
+ * the library's causal SDPA, and against closed forms; the step against branch/document
+ * permutation invariance.  Nothing in the paper prints an attention output value, so
+ * beyond those pins the numeric values themselves are parity unpinned.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ------------------------------------------------------------------------------------
+ * Algorithm 2 (Appendix, "Position ID assignment"): pos_id = range(|s|); for attribute i
+ * in order, the IDs of its tokens start(a_i)..end(a_i) (inclusive) are raised by the
+ * running offset, which then grows by K_max.  Value token k of attribute n is later given
+ * pos_id[end(a_n)] + k.
+ * ---------------------------------------------------------------------------------- */
+void hpdo_alg2_position_ids(int len_s, int n_attr, const int32_t* attr_start, const int32_t* attr_end,
+                            int k_max, int32_t* pos_id)
+{
+    for (int t = 0; t < len_s; ++t) pos_id[t] = t;
+    int offset = 0;
+    for (int i = 0; i < n_attr; ++i) {
+        for (int t = attr_start[i]; t <= attr_end[i]; ++t) pos_id[t] += offset;
+        offset += k_max;
+    }
+}
+
+/* Position ID of value token k (k = 1 is the first generated token) of attribute n. */
+int32_t hpdo_alg2_value_position(const int32_t* pos_id, const int32_t* attr_end, int n, int k)
+{
+    return pos_id[attr_end[n]] + k;
+}
+
+/* ------------------------------------------------------------------------------------
+ * Step bookkeeping.  Slots are all branches ever admitted, grouped by document in prompt
+ * order.  The step's rows are the live slots in ascending slot id (Sec. 4.3.4: finished
+ * values are pruned from the input; Sec. 4.3.6: b*J*N rows when nothing is pruned).
+ *   branch_start = position ID of the branch's first token: the document prefix occupies
+ *                  positions 0..L_d-1, so the branch starts at L_d; with pos_gap > 0 the
+ *                  j-th branch of the document is shifted by Algorithm 2's running offset
+ *                  j*pos_gap.
+ *   pos_id       = branch_start + depth (Sec. 4.3.3: IDs are the previous step's plus one).
+ *   suffix_off   = first row of the slot's slab in the branch cache (slot * cap);
+ *   suffix_len   = depth, the number of this branch's tokens cached before the step.
+ * Entries past n_active are set to -1.  Returns 0, or -1 for inconsistent arguments.
+ * ---------------------------------------------------------------------------------- */
+int hpdo_build_meta(int n_docs, int n_slots,
+                    const int32_t* doc_prefix_len, const int32_t* doc_branch_cnt,
+                    const int32_t* slot_depth, const uint8_t* slot_alive,
+                    int32_t suffix_cap, int32_t pos_gap,
+                    int32_t* doc_kv_start, int32_t* doc_slot_start, int32_t* doc_active_start,
+                    int32_t* active_slot, int32_t* doc_id, int32_t* branch_start, int32_t* pos_id,
+                    int32_t* suffix_off, int32_t* suffix_len, int32_t* n_active)
+{
+    int kv = 0, sl = 0;
+    for (int d = 0; d < n_docs; ++d) {
+        if (doc_prefix_len[d] < 0 || doc_branch_cnt[d] < 0) return -1;
+        doc_kv_start[d] = kv;   kv += doc_prefix_len[d];
+        doc_slot_start[d] = sl; sl += doc_branch_cnt[d];
+    }
+    doc_kv_start[n_docs] = kv;
+    doc_slot_start[n_docs] = sl;
+    if (sl != n_slots) return -1;
+
+    int r = 0;
+    for (int d = 0; d < n_docs; ++d) {
+        doc_active_start[d] = r;
+        for (int j = 0; j < doc_branch_cnt[d]; ++j) {
+            int s = doc_slot_start[d] + j;
+            if (!slot_alive[s]) continue;
+            active_slot[r]  = s;
+            doc_id[r]       = d;
+            branch_start[r] = doc_prefix_len[d] + j * pos_gap;
+            pos_id[r]       = branch_start[r] + slot_depth[s];
+            suffix_off[r]   = s * suffix_cap;
+            suffix_len[r]   = slot_depth[s];
+            ++r;
+        }
+    }
+    doc_active_start[n_docs] = r;
+    *n_active = r;
+    for (int i = r; i < n_slots; ++i) {
+        active_slot[i] = doc_id[i] = branch_start[i] = pos_id[i] = suffix_off[i] = suffix_len[i] = -1;
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------
+ * Rotary embedding at position `pos` for n_heads vectors of length D.  Half-split pairing:
+ * element i is paired with i + D/2; inverse frequency theta^(-2i/D); the pair is rotated by
+ * the angle pos * inv_freq:   out[i]       = x[i] cos - x[i+D/2] sin
+ *                             out[i+D/2]   = x[i+D/2] cos + x[i] sin.
+ * (The paper only says that the assigned position IDs define the positional embedding;
+ * the pairing convention is the one of the decoder families it runs.)
+ * ---------------------------------------------------------------------------------- */
+void hpdo_rope(int n_heads, int D, double theta, int32_t pos, const float* x, double* out)
+{
+    int half = D / 2;
+    for (int h = 0; h < n_heads; ++h) {
+        const float* xv = x + (size_t)h * D;
+        double* ov = out + (size_t)h * D;
+        for (int i = 0; i < half; ++i) {
+            double inv_freq = pow(theta, -2.0 * (double)i / (double)D);
+            double ang = (double)pos * inv_freq;
+            double c = cos(ang), s = sin(ang);
+            double a = (double)xv[i], b = (double)xv[i + half];
+            ov[i]        = a * c - b * s;
+            ov[i + half] = b * c + a * s;
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------------------
+ * Ordinary causal scaled-dot-product attention, one query row.  The query sits at
+ * sequence index `row` of a sequence whose keys/values are K,V[0..]; causality lets it see
+ * indices 0..row (itself included).  Grouped-query attention: q head h uses kv head
+ * h / (Hq/Hkv).  Softmax with the maximum subtracted; lse = max + log(sum).
+ *   q [Hq, D], K,V [>= row+1, Hkv, D]  ->  o [Hq, D], lse [Hq]
+ * ---------------------------------------------------------------------------------- */
+void hpdo_causal_attention_row(int row, int Hq, int Hkv, int D, double scale,
+                               const double* q, const double* K, const double* V,
+                               double* o, double* lse, double* score_scratch /* [row+1] */)
+{
+    int G = Hq / Hkv;
+    int n = row + 1;
+    for (int h = 0; h < Hq; ++h) {
+        int hk = h / G;
+        const double* qv = q + (size_t)h * D;
+        double mx = -INFINITY;
+        for (int j = 0; j < n; ++j) {
+            const double* kv = K + ((size_t)j * Hkv + hk) * D;
+            double acc = 0.0;
+            for (int d = 0; d < D; ++d) acc += qv[d] * kv[d];
+            score_scratch[j] = acc * scale;
+            if (score_scratch[j] > mx) mx = score_scratch[j];
+        }
+        double den = 0.0;
+        for (int j = 0; j < n; ++j) {
+            score_scratch[j] = exp(score_scratch[j] - mx);
+            den += score_scratch[j];
+        }
+        double* ov = o + (size_t)h * D;
+        for (int d = 0; d < D; ++d) ov[d] = 0.0;
+        for (int j = 0; j < n; ++j) {
+            const double* vv = V + ((size_t)j * Hkv + hk) * D;
+            double p = score_scratch[j] / den;
+            for (int d = 0; d < D; ++d) ov[d] += p * vv[d];
+        }
+        if (lse) lse[h] = mx + log(den);
+    }
+}
+
+/* ------------------------------------------------------------------------------------
+ * One decode step for every live branch (Eq. 5-6; Sec. 4.3.3).  For row r (document d,
+ * depth k, position pos_id[r]):
+ *   q' = rope(q[r], pos), k' = rope(k_new[r], pos);
+ *   sequence = the document's cached prefix rows, then the branch's k cached rows, then
+ *              (k', v_new[r]); its length is L_d + k + 1 and the new token is its last index;
+ *   o[r] = causal attention of q' at that last index.
+ * Cached keys are used as stored (a KV cache holds keys already rotated).
+ *   q [n_active,Hq,D], k_new,v_new [n_active,Hkv,D], prefix_k/v [sum L,Hkv,D],
+ *   suffix_k/v [n_slots*cap,Hkv,D]  ->  o [n_active,Hq,D], lse [n_active,Hq],
+ *   q_rot [n_active,Hq,D], k_rot [n_active,Hkv,D]   (outputs in fp32; lse/q_rot/k_rot may be NULL)
+ * Returns the number of threads used, or -1 on allocation failure.
+ * ---------------------------------------------------------------------------------- */
+int hpdo_decode_step(int Hq, int Hkv, int D, double theta, double scale,
+                     int n_active,
+                     const int32_t* doc_id, const int32_t* pos_id,
+                     const int32_t* suffix_off, const int32_t* suffix_len,
+                     const int32_t* doc_kv_start, const int32_t* doc_prefix_len,
+                     const float* q, const float* k_new, const float* v_new,
+                     const float* prefix_k, const float* prefix_v,
+                     const float* suffix_k, const float* suffix_v,
+                     float* o, float* lse, float* q_rot, float* k_rot,
+                     int n_threads)
+{
+    int used = 1, fail = 0;
+    size_t kvw = (size_t)Hkv * D, qw = (size_t)Hq * D;
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#endif
+#pragma omp parallel
+    {
+#ifdef _OPENMP
+#pragma omp single
+        used = omp_get_num_threads();
+#endif
+#pragma omp for schedule(dynamic, 1)
+        for (int r = 0; r < n_active; ++r) {
+            int d = doc_id[r];
+            int L = doc_prefix_len[d];
+            int k = suffix_len[r];
+            int n = L + k + 1;
+            double* Kc = (double*)malloc(sizeof(double) * (size_t)n * kvw);
+            double* Vc = (double*)malloc(sizeof(double) * (size_t)n * kvw);
+            double* qr = (double*)malloc(sizeof(double) * qw);
+            double* orow = (double*)malloc(sizeof(double) * qw);
+            double* lrow = (double*)malloc(sizeof(double) * (size_t)Hq);
+            double* sc = (double*)malloc(sizeof(double) * (size_t)n);
+            if (!Kc || !Vc || !qr || !orow || !lrow || !sc) {
+                fail = 1;
+            } else {
+                /* the concatenated sequence: prefix, own earlier tokens, the new token */
+                const float* pk = prefix_k + (size_t)doc_kv_start[d] * kvw;
+                const float* pv = prefix_v + (size_t)doc_kv_start[d] * kvw;
+                for (size_t i = 0; i < (size_t)L * kvw; ++i) { Kc[i] = pk[i]; Vc[i] = pv[i]; }
+                const float* sk = suffix_k + (size_t)suffix_off[r] * kvw;
+                const float* sv = suffix_v + (size_t)suffix_off[r] * kvw;
+                for (size_t i = 0; i < (size_t)k * kvw; ++i) {
+                    Kc[(size_t)L * kvw + i] = sk[i];
+                    Vc[(size_t)L * kvw + i] = sv[i];
+                }
+                hpdo_rope(Hkv, D, theta, pos_id[r], k_new + (size_t)r * kvw, Kc + (size_t)(L + k) * kvw);
+                for (size_t i = 0; i < kvw; ++i) Vc[(size_t)(L + k) * kvw + i] = v_new[(size_t)r * kvw + i];
+                hpdo_rope(Hq, D, theta, pos_id[r], q + (size_t)r * qw, qr);
+
+                hpdo_causal_attention_row(n - 1, Hq, Hkv, D, scale, qr, Kc, Vc, orow, lrow, sc);
+
+                for (size_t i = 0; i < qw; ++i) o[(size_t)r * qw + i] = (float)orow[i];
+                if (lse) for (int h = 0; h < Hq; ++h) lse[(size_t)r * Hq + h] = (float)lrow[h];
+                if (q_rot) for (size_t i = 0; i < qw; ++i) q_rot[(size_t)r * qw + i] = (float)qr[i];
+                if (k_rot) for (size_t i = 0; i < kvw; ++i) k_rot[(size_t)r * kvw + i] = (float)Kc[(size_t)(L + k) * kvw + i];
+            }
+            free(Kc); free(Vc); free(qr); free(orow); free(lrow); free(sc);
+        }
+    }
+    return fail ? -1 : used;
+}
+
+/* Append rule of Sec. 4.3.2 in the branch-slab layout: the step's rotated key and its value
+ * go to row suffix_off + suffix_len of the branch cache, unless the slab is full (Sec. 4.3.4:
+ * values that reach K_max are truncated).  overflow[r] = 1 marks a suppressed write. */
+void hpdo_kv_append(int Hkv, int D, int n_active, int32_t suffix_cap,
+                    const int32_t* suffix_off, const int32_t* suffix_len,
+                    const float* k_rot, const float* v_new,
+                    float* suffix_k, float* suffix_v, uint8_t* overflow)
+{
+    size_t kvw = (size_t)Hkv * D;
+    for (int r = 0; r < n_active; ++r) {
+        if (suffix_len[r] >= suffix_cap) { if (overflow) overflow[r] = 1; continue; }
+        if (overflow) overflow[r] = 0;
+        size_t dst = ((size_t)suffix_off[r] + (size_t)suffix_len[r]) * kvw;
+        memcpy(suffix_k + dst, k_rot + (size_t)r * kvw, kvw * sizeof(float));
+        memcpy(suffix_v + dst, v_new + (size_t)r * kvw, kvw * sizeof(float));
+    }
+}
