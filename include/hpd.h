@@ -1,0 +1,166 @@
+/*
+ * libhpd -- decode-step attention of Hyper-Parallel Decoding (HPD) for NVIDIA B200 (sm_100a).
+ *
+ * HPD decodes many attribute values of many stacked documents in parallel: every live
+ * "branch" (one value being generated) contributes ONE new token per decode step, and that
+ * token may depend on its document and on the branch's own earlier tokens only (Eq. 4-6).
+ * New tokens are appended to the KV cache out of logical order; position IDs, not memory
+ * order, say where a token sits (Sec. 4.3.1-4.3.3).
+ *
+ * Conventions for every entry point
+ *   - plain C ABI; returns 0 (HPD_OK) or a negative HPD_E_* code; nothing throws.
+ *   - "dev" pointers are CUDA device memory owned by the caller; "host" pointers are ordinary
+ *     host memory.  The library allocates no device memory.  Pointers to bf16 tensors must be
+ *     16-byte aligned; the innermost dimension is contiguous; tensors are dense row-major
+ *     with the shapes stated.
+ *   - every call only ENQUEUES work on `stream` (a cudaStream_t passed as void*) and never
+ *     synchronises.  Sizes that change per step (n_active) are read on the device.
+ *   - problems detected on the device set bits (HPD_S_*) in the caller's `dev_status` word
+ *     with the offending access suppressed; kernels never trap.
+ *   - documents are numbered globally in prompt order; "slots" are all branches ever admitted,
+ *     numbered globally and grouped by document; "rows" are the live slots of this step in
+ *     ascending slot id.  G = Hq / Hkv.
+ *   - call order of one step:  hpd_build_meta  (once per step)
+ *                              per layer: hpd_rope -> hpd_kv_append -> hpd_attn_decode.
+ */
+#ifndef HPD_H_
+#define HPD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Attention geometry.  Supported: D in {64, 128}; Hq % Hkv == 0 with G in {1, 2, 4, 8};
+ * 1 <= suffix_cap.  sm_scale multiplies q.k before the softmax (1/sqrt(D) in the paper's
+ * "scaled dot-product attention", Sec. 4.3.2).  suffix_cap is the branch-cache slab size in
+ * tokens: the K_max of Sec. 4.3.1 (values longer than K_max are truncated, Sec. 4.3.4). */
+typedef struct hpd_geom {
+    int32_t Hq, Hkv, D;
+    float   rope_theta, sm_scale;
+    int32_t suffix_cap;
+} hpd_geom;
+
+enum {
+    HPD_OK          =  0,
+    HPD_E_ARG       = -1,   /* null / misaligned pointer, negative size                        */
+    HPD_E_GEOM      = -2,   /* geometry outside the supported set                              */
+    HPD_E_WORKSPACE = -3,   /* workspace_bytes smaller than hpd_workspace_bytes() reports      */
+    HPD_E_CAPACITY  = -4,   /* a size exceeds what the call can index (int32 tables)           */
+    HPD_E_CUDA      = -5    /* a CUDA runtime/driver call failed; see hpd_last_cuda_error()    */
+};
+
+/* bits of *dev_status */
+enum {
+    HPD_S_OVERFLOW  = 1,    /* hpd_kv_append: a branch slab was full, its write was suppressed */
+    HPD_S_BAD_TABLE = 2,    /* a table entry pointed outside its tensor; the row was skipped   */
+    HPD_S_TIMEOUT   = 4     /* an in-kernel wait on the kernel's own copies gave up            */
+};
+
+const char* hpd_strerror(int code);
+/* cudaError_t (as int) of the last failing CUDA call made by this library on this thread. */
+int hpd_last_cuda_error(void);
+
+/* Bytes of workspace that hpd_build_meta + hpd_attn_decode need for problems up to the given
+ * sizes.  The SAME workspace must be passed to hpd_build_meta and to the hpd_attn_decode calls
+ * of that step: build_meta leaves its split-KV work list there. */
+size_t hpd_workspace_bytes(const hpd_geom* geom /*host*/, int max_docs, int max_slots, int max_prefix_tokens);
+
+/*
+ * hpd_build_meta -- per-step bookkeeping as int32 device tables (Algorithm 2; Sec. 4.3.2-4.3.6).
+ *
+ * Inputs (dev):  doc_prefix_len[n_docs]  tokens of each document's shared prefix (L_d)
+ *                doc_branch_cnt[n_docs]  slots of each document (sum = n_slots)
+ *                slot_depth[n_slots]     branch tokens cached before this step
+ *                slot_alive[n_slots]     non-zero while the branch is still decoding (pruning, Sec. 4.3.4)
+ *                pos_gap                 0: positions continue the document, pos = L_d + depth;
+ *                                        K_max: the j-th branch of a document is shifted by
+ *                                        Algorithm 2's running offset j*K_max
+ * Outputs (dev): doc_kv_start[n_docs+1]      exclusive scan of doc_prefix_len
+ *                doc_slot_start[n_docs+1]    exclusive scan of doc_branch_cnt
+ *                doc_active_start[n_docs+1]  CSR of rows per document
+ *                per row r < n_active (arrays of n_slots entries, the rest set to -1):
+ *                active_slot[r]  slot id (ascending)      doc_id[r]      its document
+ *                branch_start[r] position ID of the branch's first token
+ *                pos_id[r]       branch_start + depth (Sec. 4.3.3: previous ID + 1)
+ *                suffix_off[r]   first row of the slot's slab in the branch cache (slot*suffix_cap)
+ *                suffix_len[r]   depth
+ *                n_active[1]     number of rows
+ * Also writes the internal work list of hpd_attn_decode into `workspace`.
+ * All tables are int32 and are reproducible bit for bit.  n_docs or n_slots may be 0.
+ */
+int hpd_build_meta(const hpd_geom* geom /*host*/, int n_docs, int n_slots,
+                   const int32_t* doc_prefix_len, const int32_t* doc_branch_cnt,
+                   const int32_t* slot_depth, const uint8_t* slot_alive, int32_t pos_gap,
+                   int32_t* doc_kv_start, int32_t* doc_slot_start, int32_t* doc_active_start,
+                   int32_t* active_slot, int32_t* doc_id, int32_t* branch_start, int32_t* pos_id,
+                   int32_t* suffix_off, int32_t* suffix_len, int32_t* n_active,
+                   void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream);
+
+/*
+ * hpd_rope -- rotary embedding of the step's new q and k at each row's position ID, in place
+ * (Sec. 4.3.1: the assigned position IDs define the positional embedding; Sec. 4.4).
+ * Pairing is half-split: element i with i + D/2; angle = pos_id[r] * rope_theta^(-2i/D),
+ * evaluated in fp64, rotation in fp32, result rounded to bf16 (nearest even).
+ *   q [max_rows, Hq, D] bf16 dev, k_new [max_rows, Hkv, D] bf16 dev; rows >= *n_active untouched.
+ */
+int hpd_rope(const hpd_geom* geom /*host*/, int max_rows, const int32_t* n_active /*dev*/,
+             const int32_t* pos_id /*dev*/, void* q, void* k_new, void* stream);
+
+/*
+ * hpd_kv_append -- append each row's (rotated) key and its value to the branch cache
+ * (Sec. 4.3.2: new tokens are appended to the cache; here every slot owns a slab of
+ * suffix_cap rows, row suffix_off[r] + suffix_len[r] receives the token).
+ *   k_new, v_new [max_rows, Hkv, D] bf16 dev;  suffix_k, suffix_v [n_slots*suffix_cap, Hkv, D] bf16 dev.
+ * A full slab (suffix_len >= suffix_cap) gets no write and sets HPD_S_OVERFLOW.
+ * The caller advances slot_depth for the next step.
+ */
+int hpd_kv_append(const hpd_geom* geom /*host*/, int max_rows, int n_slots, const int32_t* n_active,
+                  const int32_t* suffix_off, const int32_t* suffix_len,
+                  const void* k_new, const void* v_new, void* suffix_k, void* suffix_v,
+                  int32_t* dev_status, void* stream);
+
+/*
+ * hpd_attn_decode -- the HPD decode attention (Eq. 5-6; Sec. 4.3.3).  For row r (document d,
+ * slot s) and q head h:   o = softmax(sm_scale * q . [K_prefix(d) ; K_suffix(s)]^T) [V_prefix(d) ; V_suffix(s)]
+ * over the document's L_d prefix tokens and the branch's own cached tokens.  The prefix of a
+ * document is read from memory once per KV head for all of the document's rows.
+ *   q [max_rows, Hq, D] bf16 (already rotated); prefix_k/v [total_prefix_tokens, Hkv, D] bf16
+ *   (as cached, i.e. rotated); suffix_k/v [n_slots*suffix_cap, Hkv, D] bf16; tables from
+ *   hpd_build_meta; suffix_includes_new = 1 when hpd_kv_append already ran this step (the branch
+ *   then sees suffix_len+1 cached tokens, the new token among them), 0 to see suffix_len tokens.
+ *   o [max_rows, Hq, D] bf16; lse [max_rows, Hq] fp32 natural-log sum-exp of the scaled scores,
+ *   may be NULL.  Rows >= *n_active are not written.  A row with no visible token yields o = 0,
+ *   lse = -inf.
+ */
+int hpd_attn_decode(const hpd_geom* geom /*host*/, int n_docs, int max_rows, int n_slots, int total_prefix_tokens,
+                    const void* q, const void* prefix_k, const void* prefix_v,
+                    const void* suffix_k, const void* suffix_v,
+                    const int32_t* doc_kv_start, const int32_t* doc_prefix_len, const int32_t* doc_active_start,
+                    const int32_t* doc_id, const int32_t* suffix_off, const int32_t* suffix_len,
+                    const int32_t* n_active, int suffix_includes_new,
+                    void* o, float* lse,
+                    void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream);
+
+/*
+ * std_attn_decode -- the in-repo comparison: standard batched decode in which every branch is a
+ * sequence of its own with a private physical copy of [prefix ; branch tokens] (parallel streams
+ * as batch elements, Sec. 2; standard batched inference, Sec. 4.3.6).  Same math as
+ * hpd_attn_decode on the same tokens, GQA, split-KV.
+ *   q [max_rows, Hq, D] bf16 (rotated); dup_k/v [total_tokens, Hkv, D] bf16;
+ *   seq_start [max_rows] int64 first token row of each sequence; seq_len [max_rows] int32;
+ *   o [max_rows, Hq, D] bf16; lse nullable.
+ * workspace: std_workspace_bytes(); may be NULL when that reports 0.
+ */
+size_t std_workspace_bytes(const hpd_geom* geom /*host*/, int max_rows, int max_seq_len);
+int std_attn_decode(const hpd_geom* geom /*host*/, int max_rows, int max_seq_len, const int32_t* n_active,
+                    const void* q, const void* dup_k, const void* dup_v,
+                    const int64_t* seq_start, const int32_t* seq_len,
+                    void* o, float* lse, void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HPD_H_ */

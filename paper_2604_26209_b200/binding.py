@@ -1,0 +1,170 @@
+"""Thin Python binding of ``libhpd.so`` (C ABI declared in ``include/hpd.h``).
+
+Argument marshalling only: tensors are passed as raw device pointers together with the current
+CUDA stream; every step of the path runs in the library's kernels.  PyTorch is used for device
+memory and streams.  The library must be present -- there is no fallback; ``load()`` raises if
+``libhpd.so`` has not been built (``python -m paper_2604_26209_b200.build``).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libhpd.so")
+
+EXPORTS = ("hpd_strerror", "hpd_last_cuda_error", "hpd_workspace_bytes", "hpd_build_meta", "hpd_rope",
+           "hpd_kv_append", "hpd_attn_decode", "std_workspace_bytes", "std_attn_decode")
+
+HPD_S_OVERFLOW, HPD_S_BAD_TABLE, HPD_S_TIMEOUT = 1, 2, 4
+
+
+class HpdGeom(C.Structure):
+    _fields_ = [("Hq", C.c_int32), ("Hkv", C.c_int32), ("D", C.c_int32), ("rope_theta", C.c_float),
+                ("sm_scale", C.c_float), ("suffix_cap", C.c_int32)]
+
+
+class HpdError(RuntimeError):
+    pass
+
+
+_lib = None
+
+
+def load() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise HpdError(f"{LIB_PATH} is missing: build it with `python -m paper_2604_26209_b200.build` "
+                           "(there is no CPU fallback)")
+        lib = C.CDLL(LIB_PATH)
+        lib.hpd_strerror.restype = C.c_char_p
+        lib.hpd_strerror.argtypes = [C.c_int]
+        lib.hpd_last_cuda_error.restype = C.c_int
+        lib.hpd_workspace_bytes.restype = C.c_size_t
+        lib.hpd_workspace_bytes.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int, C.c_int]
+        lib.std_workspace_bytes.restype = C.c_size_t
+        lib.std_workspace_bytes.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int]
+        vp = C.c_void_p
+        lib.hpd_build_meta.restype = C.c_int
+        lib.hpd_build_meta.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int, vp, vp, vp, vp, C.c_int32] + [vp] * 10 + \
+                                      [vp, C.c_size_t, vp, vp]
+        lib.hpd_rope.restype = C.c_int
+        lib.hpd_rope.argtypes = [C.POINTER(HpdGeom), C.c_int, vp, vp, vp, vp, vp]
+        lib.hpd_kv_append.restype = C.c_int
+        lib.hpd_kv_append.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int] + [vp] * 9
+        lib.hpd_attn_decode.restype = C.c_int
+        lib.hpd_attn_decode.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int, C.c_int, C.c_int] + [vp] * 12 + \
+                                       [C.c_int, vp, vp, vp, C.c_size_t, vp, vp]
+        lib.std_attn_decode.restype = C.c_int
+        lib.std_attn_decode.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int] + [vp] * 8 + [vp, C.c_size_t, vp]
+        _lib = lib
+    return _lib
+
+
+def make_geom(g) -> HpdGeom:
+    return HpdGeom(int(g.Hq), int(g.Hkv), int(g.D), float(g.rope_theta), float(g.sm_scale), int(g.suffix_cap))
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device-resident contiguous tensors only"
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        lib = load()
+        msg = lib.hpd_strerror(rc).decode()
+        if rc == -5:
+            msg += f" [cudaError {lib.hpd_last_cuda_error()}]"
+        raise HpdError(f"{what}: {msg} ({rc})")
+
+
+def hpd_workspace_bytes(geom, max_docs: int, max_slots: int, max_prefix_tokens: int) -> int:
+    g = make_geom(geom)
+    return int(load().hpd_workspace_bytes(C.byref(g), max_docs, max_slots, max_prefix_tokens))
+
+
+def std_workspace_bytes(geom, max_rows: int, max_seq_len: int) -> int:
+    g = make_geom(geom)
+    return int(load().std_workspace_bytes(C.byref(g), max_rows, max_seq_len))
+
+
+@dataclass
+class MetaTables:
+    """Device int32 tables written by ``hpd_build_meta`` (plus the workspace and status word)."""
+    doc_kv_start: torch.Tensor
+    doc_slot_start: torch.Tensor
+    doc_active_start: torch.Tensor
+    active_slot: torch.Tensor
+    doc_id: torch.Tensor
+    branch_start: torch.Tensor
+    pos_id: torch.Tensor
+    suffix_off: torch.Tensor
+    suffix_len: torch.Tensor
+    n_active: torch.Tensor
+    workspace: torch.Tensor
+    dev_status: torch.Tensor
+
+    NAMES = ("doc_kv_start", "doc_slot_start", "doc_active_start", "active_slot", "doc_id", "branch_start",
+             "pos_id", "suffix_off", "suffix_len")
+
+    @staticmethod
+    def alloc(geom, n_docs: int, n_slots: int, total_prefix: int, device="cuda") -> "MetaTables":
+        i32 = lambda n: torch.empty(max(n, 1), dtype=torch.int32, device=device)
+        ws = torch.empty(max(hpd_workspace_bytes(geom, n_docs, n_slots, total_prefix), 256), dtype=torch.uint8, device=device)
+        return MetaTables(i32(n_docs + 1), i32(n_docs + 1), i32(n_docs + 1), *[i32(n_slots) for _ in range(6)],
+                          torch.zeros(1, dtype=torch.int32, device=device), ws,
+                          torch.zeros(1, dtype=torch.int32, device=device))
+
+
+def hpd_build_meta(geom, n_docs, n_slots, doc_prefix_len, doc_branch_cnt, slot_depth, slot_alive, pos_gap, m: MetaTables):
+    g = make_geom(geom)
+    rc = load().hpd_build_meta(C.byref(g), n_docs, n_slots, _ptr(doc_prefix_len), _ptr(doc_branch_cnt), _ptr(slot_depth),
+                               _ptr(slot_alive), int(pos_gap), _ptr(m.doc_kv_start), _ptr(m.doc_slot_start),
+                               _ptr(m.doc_active_start), _ptr(m.active_slot), _ptr(m.doc_id), _ptr(m.branch_start),
+                               _ptr(m.pos_id), _ptr(m.suffix_off), _ptr(m.suffix_len), _ptr(m.n_active),
+                               _ptr(m.workspace), m.workspace.numel(), _ptr(m.dev_status), _stream())
+    _check(rc, "hpd_build_meta")
+
+
+def hpd_rope(geom, max_rows, n_active, pos_id, q, k_new):
+    g = make_geom(geom)
+    _check(load().hpd_rope(C.byref(g), max_rows, _ptr(n_active), _ptr(pos_id), _ptr(q), _ptr(k_new), _stream()), "hpd_rope")
+
+
+def hpd_kv_append(geom, max_rows, n_slots, n_active, suffix_off, suffix_len, k_new, v_new, suffix_k, suffix_v, dev_status):
+    g = make_geom(geom)
+    rc = load().hpd_kv_append(C.byref(g), max_rows, n_slots, _ptr(n_active), _ptr(suffix_off), _ptr(suffix_len),
+                              _ptr(k_new), _ptr(v_new), _ptr(suffix_k), _ptr(suffix_v), _ptr(dev_status), _stream())
+    _check(rc, "hpd_kv_append")
+
+
+def hpd_attn_decode(geom, n_docs, max_rows, n_slots, total_prefix_tokens, q, prefix_k, prefix_v, suffix_k, suffix_v,
+                    doc_prefix_len, m: MetaTables, suffix_includes_new, o, lse=None):
+    g = make_geom(geom)
+    rc = load().hpd_attn_decode(C.byref(g), n_docs, max_rows, n_slots, total_prefix_tokens, _ptr(q), _ptr(prefix_k),
+                                _ptr(prefix_v), _ptr(suffix_k), _ptr(suffix_v), _ptr(m.doc_kv_start),
+                                _ptr(doc_prefix_len), _ptr(m.doc_active_start), _ptr(m.doc_id), _ptr(m.suffix_off),
+                                _ptr(m.suffix_len), _ptr(m.n_active), int(bool(suffix_includes_new)), _ptr(o), _ptr(lse),
+                                _ptr(m.workspace), m.workspace.numel(), _ptr(m.dev_status), _stream())
+    _check(rc, "hpd_attn_decode")
+
+
+def std_attn_decode(geom, max_rows, max_seq_len, n_active, q, dup_k, dup_v, seq_start, seq_len, o, lse=None,
+                    workspace=None):
+    g = make_geom(geom)
+    wsb = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = load().std_attn_decode(C.byref(g), max_rows, max_seq_len, _ptr(n_active), _ptr(q), _ptr(dup_k), _ptr(dup_v),
+                                _ptr(seq_start), _ptr(seq_len), _ptr(o), _ptr(lse), _ptr(workspace), wsb, _stream())
+    _check(rc, "std_attn_decode")

@@ -1,0 +1,230 @@
+// extern "C" entry points of libhpd (see include/hpd.h): argument checks and kernel dispatch only.
+#include <cstdlib>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace hpd {
+
+static thread_local int g_last_cuda_error = 0;
+void set_last_cuda_error(cudaError_t e) { g_last_cuda_error = static_cast<int>(e); }
+
+int geom_check(const hpd_geom* g)
+{
+    if (!g) return HPD_E_ARG;
+    if (g->D != 64 && g->D != 128) return HPD_E_GEOM;
+    if (g->Hq <= 0 || g->Hkv <= 0 || g->Hq % g->Hkv != 0) return HPD_E_GEOM;
+    const int G = g->Hq / g->Hkv;
+    if (G != 1 && G != 2 && G != 4 && G != 8) return HPD_E_GEOM;
+    if (g->suffix_cap < 1) return HPD_E_GEOM;
+    if (!(g->rope_theta > 0.f)) return HPD_E_GEOM;
+    return HPD_OK;
+}
+
+int sm_count()
+{
+    static int cached = 0;
+    if (cached > 0) return cached;
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) {
+        cached = n;
+        return n;
+    }
+    (void)cudaGetLastError();
+    return 148;
+}
+
+// HPD_ATTN_IMPL=simt forces the scalar kernel in hpd_attn_decode (debugging aid).
+static bool force_simt()
+{
+    static int v = -1;
+    if (v < 0) {
+        const char* e = std::getenv("HPD_ATTN_IMPL");
+        v = (e && std::strcmp(e, "simt") == 0) ? 1 : 0;
+    }
+    return v == 1;
+}
+
+}  // namespace hpd
+
+using namespace hpd;
+
+extern "C" {
+
+const char* hpd_strerror(int code)
+{
+    switch (code) {
+        case HPD_OK: return "ok";
+        case HPD_E_ARG: return "invalid argument (null or misaligned pointer, negative size)";
+        case HPD_E_GEOM: return "unsupported geometry (need D in {64,128}, Hq/Hkv in {1,2,4,8}, suffix_cap >= 1)";
+        case HPD_E_WORKSPACE: return "workspace too small";
+        case HPD_E_CAPACITY: return "size exceeds int32 table range";
+        case HPD_E_CUDA: return "CUDA call failed (see hpd_last_cuda_error)";
+        default: return "unknown error code";
+    }
+}
+
+int hpd_last_cuda_error(void) { return g_last_cuda_error; }
+
+size_t hpd_workspace_bytes(const hpd_geom* geom, int max_docs, int max_slots, int /*max_prefix_tokens*/)
+{
+    if (geom_check(geom) != HPD_OK || max_docs < 0 || max_slots < 0) return 0;
+    return ws_layout(*geom, max_docs, max_slots, sm_count()).total;
+}
+
+int hpd_build_meta(const hpd_geom* geom, int n_docs, int n_slots,
+                   const int32_t* doc_prefix_len, const int32_t* doc_branch_cnt,
+                   const int32_t* slot_depth, const uint8_t* slot_alive, int32_t pos_gap,
+                   int32_t* doc_kv_start, int32_t* doc_slot_start, int32_t* doc_active_start,
+                   int32_t* active_slot, int32_t* doc_id, int32_t* branch_start, int32_t* pos_id,
+                   int32_t* suffix_off, int32_t* suffix_len, int32_t* n_active,
+                   void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream)
+{
+    int rc = geom_check(geom);
+    if (rc != HPD_OK) return rc;
+    if (n_docs < 0 || n_slots < 0 || pos_gap < 0) return HPD_E_ARG;
+    if (n_docs == 0 && n_slots > 0) return HPD_E_ARG;
+    if (!doc_kv_start || !doc_slot_start || !doc_active_start || !n_active || !workspace) return HPD_E_ARG;
+    if (n_docs > 0 && (!doc_prefix_len || !doc_branch_cnt)) return HPD_E_ARG;
+    if (n_slots > 0 && (!slot_depth || !slot_alive || !active_slot || !doc_id || !branch_start || !pos_id ||
+                        !suffix_off || !suffix_len)) return HPD_E_ARG;
+    if (static_cast<long long>(n_slots) * geom->suffix_cap > 0x7fffffffll) return HPD_E_CAPACITY;
+    if (!aligned16(workspace)) return HPD_E_ARG;
+    const int n_sm = sm_count();
+    const WsLayout lay = ws_layout(*geom, n_docs, n_slots, n_sm);
+    if (workspace_bytes < lay.total) return HPD_E_WORKSPACE;
+    return launch_build_meta(*geom, n_docs, n_slots, doc_prefix_len, doc_branch_cnt, slot_depth, slot_alive, pos_gap,
+                             doc_kv_start, doc_slot_start, doc_active_start, active_slot, doc_id, branch_start, pos_id,
+                             suffix_off, suffix_len, n_active, workspace, lay, n_sm, dev_status,
+                             static_cast<cudaStream_t>(stream));
+}
+
+int hpd_rope(const hpd_geom* geom, int max_rows, const int32_t* n_active, const int32_t* pos_id,
+             void* q, void* k_new, void* stream)
+{
+    int rc = geom_check(geom);
+    if (rc != HPD_OK) return rc;
+    if (max_rows < 0) return HPD_E_ARG;
+    if (max_rows == 0) return HPD_OK;
+    if (!n_active || !pos_id || !q || !k_new || !aligned16(q) || !aligned16(k_new)) return HPD_E_ARG;
+    return launch_rope(*geom, max_rows, n_active, pos_id, static_cast<__nv_bfloat16*>(q),
+                       static_cast<__nv_bfloat16*>(k_new), static_cast<cudaStream_t>(stream));
+}
+
+int hpd_kv_append(const hpd_geom* geom, int max_rows, int n_slots, const int32_t* n_active,
+                  const int32_t* suffix_off, const int32_t* suffix_len,
+                  const void* k_new, const void* v_new, void* suffix_k, void* suffix_v,
+                  int32_t* dev_status, void* stream)
+{
+    int rc = geom_check(geom);
+    if (rc != HPD_OK) return rc;
+    if (max_rows < 0 || n_slots < 0) return HPD_E_ARG;
+    if (max_rows == 0) return HPD_OK;
+    if (!n_active || !suffix_off || !suffix_len || !k_new || !v_new || !suffix_k || !suffix_v) return HPD_E_ARG;
+    if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(suffix_k) || !aligned16(suffix_v)) return HPD_E_ARG;
+    return launch_kv_append(*geom, max_rows, n_slots, n_active, suffix_off, suffix_len,
+                            static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
+                            static_cast<__nv_bfloat16*>(suffix_k), static_cast<__nv_bfloat16*>(suffix_v), dev_status,
+                            static_cast<cudaStream_t>(stream));
+}
+
+int hpd_attn_decode(const hpd_geom* geom, int n_docs, int max_rows, int n_slots, int total_prefix_tokens,
+                    const void* q, const void* prefix_k, const void* prefix_v,
+                    const void* suffix_k, const void* suffix_v,
+                    const int32_t* doc_kv_start, const int32_t* doc_prefix_len, const int32_t* doc_active_start,
+                    const int32_t* doc_id, const int32_t* suffix_off, const int32_t* suffix_len,
+                    const int32_t* n_active, int suffix_includes_new,
+                    void* o, float* lse,
+                    void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream)
+{
+    int rc = geom_check(geom);
+    if (rc != HPD_OK) return rc;
+    if (n_docs < 0 || max_rows < 0 || n_slots < 0 || total_prefix_tokens < 0) return HPD_E_ARG;
+    if (max_rows == 0 || n_docs == 0) return HPD_OK;
+    if (!q || !suffix_k || !suffix_v || !doc_kv_start || !doc_prefix_len || !doc_active_start || !doc_id ||
+        !suffix_off || !suffix_len || !n_active || !o || !workspace) return HPD_E_ARG;
+    if (total_prefix_tokens > 0 && (!prefix_k || !prefix_v)) return HPD_E_ARG;
+    if (!aligned16(q) || !aligned16(prefix_k) || !aligned16(prefix_v) || !aligned16(suffix_k) ||
+        !aligned16(suffix_v) || !aligned16(o) || !aligned16(workspace)) return HPD_E_ARG;
+    const WsLayout lay = ws_layout(*geom, n_docs, n_slots, sm_count());
+    if (workspace_bytes < lay.total) return HPD_E_WORKSPACE;
+
+    if (!force_simt()) {
+        AttnArgs a{};
+        a.g = *geom;
+        a.n_docs = n_docs; a.max_rows = max_rows; a.n_slots = n_slots; a.total_prefix = total_prefix_tokens;
+        a.q = static_cast<const __nv_bfloat16*>(q);
+        a.prefix_k = static_cast<const __nv_bfloat16*>(prefix_k);
+        a.prefix_v = static_cast<const __nv_bfloat16*>(prefix_v);
+        a.suffix_k = static_cast<const __nv_bfloat16*>(suffix_k);
+        a.suffix_v = static_cast<const __nv_bfloat16*>(suffix_v);
+        a.doc_kv_start = doc_kv_start; a.doc_prefix_len = doc_prefix_len; a.doc_active_start = doc_active_start;
+        a.doc_id = doc_id; a.suffix_off = suffix_off; a.suffix_len = suffix_len; a.n_active = n_active;
+        a.suffix_extra = suffix_includes_new ? 1 : 0;
+        a.o = static_cast<__nv_bfloat16*>(o);
+        a.lse = lse;
+        a.workspace = workspace; a.lay = lay; a.dev_status = dev_status;
+        a.stream = static_cast<cudaStream_t>(stream);
+        return launch_attn_tc(a);
+    }
+    SimtArgs s{};
+    s.g = *geom;
+    s.max_rows = max_rows; s.n_splits = 1; s.n_active = n_active;
+    s.q = static_cast<const __nv_bfloat16*>(q);
+    s.k1 = static_cast<const __nv_bfloat16*>(prefix_k); s.v1 = static_cast<const __nv_bfloat16*>(prefix_v);
+    s.doc_id = doc_id; s.doc_kv_start = doc_kv_start; s.doc_prefix_len = doc_prefix_len;
+    s.k2 = static_cast<const __nv_bfloat16*>(suffix_k); s.v2 = static_cast<const __nv_bfloat16*>(suffix_v);
+    s.suffix_off = suffix_off; s.suffix_len = suffix_len; s.suffix_extra = suffix_includes_new ? 1 : 0;
+    s.o = static_cast<__nv_bfloat16*>(o); s.lse = lse; s.part = nullptr;
+    s.stream = static_cast<cudaStream_t>(stream);
+    return launch_attn_simt(s);
+}
+
+static int std_splits(const hpd_geom* g, int max_rows, int max_seq_len)
+{
+    // enough warps to fill the machine: split long sequences when the batch is small
+    const long long warps = static_cast<long long>(max_rows) * g->Hkv;
+    const long long target = static_cast<long long>(sm_count()) * 32;
+    if (warps <= 0 || warps >= target) return 1;
+    long long s = (target + warps - 1) / warps;
+    const long long by_len = max_seq_len / 256;       // at least 256 keys per split
+    if (s > by_len) s = by_len;
+    if (s > 32) s = 32;
+    return s < 1 ? 1 : static_cast<int>(s);
+}
+
+size_t std_workspace_bytes(const hpd_geom* geom, int max_rows, int max_seq_len)
+{
+    if (geom_check(geom) != HPD_OK || max_rows <= 0) return 0;
+    const int s = std_splits(geom, max_rows, max_seq_len);
+    if (s <= 1) return 0;
+    return sizeof(float) * static_cast<size_t>(max_rows) * geom->Hq * s * (geom->D + 2);
+}
+
+int std_attn_decode(const hpd_geom* geom, int max_rows, int max_seq_len, const int32_t* n_active,
+                    const void* q, const void* dup_k, const void* dup_v,
+                    const int64_t* seq_start, const int32_t* seq_len,
+                    void* o, float* lse, void* workspace, size_t workspace_bytes, void* stream)
+{
+    int rc = geom_check(geom);
+    if (rc != HPD_OK) return rc;
+    if (max_rows < 0 || max_seq_len < 0) return HPD_E_ARG;
+    if (max_rows == 0) return HPD_OK;
+    if (!n_active || !q || !dup_k || !dup_v || !seq_start || !seq_len || !o) return HPD_E_ARG;
+    if (!aligned16(q) || !aligned16(dup_k) || !aligned16(dup_v) || !aligned16(o)) return HPD_E_ARG;
+    const int splits = std_splits(geom, max_rows, max_seq_len);
+    const size_t need = std_workspace_bytes(geom, max_rows, max_seq_len);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return HPD_E_WORKSPACE;
+    SimtArgs s{};
+    s.g = *geom;
+    s.max_rows = max_rows; s.n_splits = splits; s.n_active = n_active;
+    s.q = static_cast<const __nv_bfloat16*>(q);
+    s.k1 = static_cast<const __nv_bfloat16*>(dup_k); s.v1 = static_cast<const __nv_bfloat16*>(dup_v);
+    s.seq_start = seq_start; s.seq_len = seq_len;
+    s.o = static_cast<__nv_bfloat16*>(o); s.lse = lse; s.part = static_cast<float*>(workspace);
+    s.stream = static_cast<cudaStream_t>(stream);
+    return launch_attn_simt(s);
+}
+
+}  // extern "C"

@@ -1,0 +1,338 @@
+// hpd_build_meta: per-step int32 bookkeeping tables and the attention work list (device side).
+//
+// Three small kernels, all on the caller's stream, no host synchronisation:
+//   doc_scan_kernel   exclusive scans over documents (prefix tokens, slots)
+//   compact_kernel    stable compaction of live slots -> row tables, rows-per-document CSR
+//   plan_kernel       split-KV policy + work list for the attention kernel; -1 fill of table tails
+#include "common.cuh"
+
+namespace hpd {
+
+namespace {
+
+constexpr int kScanThreads = 1024;
+constexpr int kCompactThreads = 256;
+constexpr int kPlanThreads = 1024;
+
+__device__ __forceinline__ int warp_incl_scan(int v) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += t;
+    }
+    return v;
+}
+
+// Block-wide exclusive scan of one int per thread; returns the exclusive prefix and the block total.
+template <int THREADS>
+__device__ __forceinline__ int block_excl_scan(int v, int* smem /* THREADS/32 + 1 */, int& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = warp_incl_scan(v);
+    if (lane == 31) smem[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int w = (lane < THREADS / 32) ? smem[lane] : 0;
+        int wi = warp_incl_scan(w);
+        if (lane < THREADS / 32) smem[lane] = wi - w;
+        if (lane == 31) smem[THREADS / 32] = wi;
+    }
+    __syncthreads();
+    int res = incl - v + smem[warp];
+    total = smem[THREADS / 32];
+    __syncthreads();
+    return res;
+}
+
+__global__ void __launch_bounds__(kScanThreads)
+doc_scan_kernel(int n_docs, const int32_t* __restrict__ doc_prefix_len, const int32_t* __restrict__ doc_branch_cnt,
+                int32_t* __restrict__ doc_kv_start, int32_t* __restrict__ doc_slot_start)
+{
+    __shared__ int sm[kScanThreads / 32 + 1];
+    int run_kv = 0, run_sl = 0;
+    for (int base = 0; base < n_docs; base += kScanThreads) {
+        int d = base + threadIdx.x;
+        int l = d < n_docs ? doc_prefix_len[d] : 0;
+        int c = d < n_docs ? doc_branch_cnt[d] : 0;
+        int tot;
+        int el = block_excl_scan<kScanThreads>(l, sm, tot);
+        int tl = tot;
+        int ec = block_excl_scan<kScanThreads>(c, sm, tot);
+        if (d < n_docs) {
+            doc_kv_start[d] = run_kv + el;
+            doc_slot_start[d] = run_sl + ec;
+        }
+        run_kv += tl;
+        run_sl += tot;
+    }
+    if (threadIdx.x == 0) {
+        doc_kv_start[n_docs] = run_kv;
+        doc_slot_start[n_docs] = run_sl;
+    }
+}
+
+// Each block owns kCompactThreads consecutive slots.  The number of live slots before the block is
+// recounted by the block itself (reads at most n_slots bytes from L2), which keeps the kernel free of
+// any inter-block dependency.
+__global__ void __launch_bounds__(kCompactThreads)
+compact_kernel(int n_docs, int n_slots, int32_t suffix_cap, int32_t pos_gap,
+               const int32_t* __restrict__ doc_prefix_len, const int32_t* __restrict__ doc_branch_cnt,
+               const int32_t* __restrict__ doc_slot_start,
+               const int32_t* __restrict__ slot_depth, const uint8_t* __restrict__ slot_alive,
+               int32_t* __restrict__ doc_active_start, int32_t* __restrict__ active_slot,
+               int32_t* __restrict__ doc_id, int32_t* __restrict__ branch_start, int32_t* __restrict__ pos_id,
+               int32_t* __restrict__ suffix_off, int32_t* __restrict__ suffix_len, int32_t* __restrict__ n_active)
+{
+    __shared__ int sm[kCompactThreads / 32 + 1];
+    const int first = blockIdx.x * kCompactThreads;
+
+    // live slots in [0, first)
+    int cnt = 0;
+    {
+        const uintptr_t addr = reinterpret_cast<uintptr_t>(slot_alive);
+        int head = static_cast<int>((16 - (addr & 15)) & 15);
+        if (head > first) head = first;
+        for (int i = threadIdx.x; i < head; i += kCompactThreads) cnt += slot_alive[i] != 0;
+        const int n_vec = (first - head) / 16;
+        const uint4* v = reinterpret_cast<const uint4*>(slot_alive + head);
+        for (int i = threadIdx.x; i < n_vec; i += kCompactThreads) {
+            uint4 w = v[i];
+            cnt += __popc(__vcmpne4(w.x, 0u) & 0x01010101u) + __popc(__vcmpne4(w.y, 0u) & 0x01010101u) +
+                   __popc(__vcmpne4(w.z, 0u) & 0x01010101u) + __popc(__vcmpne4(w.w, 0u) & 0x01010101u);
+        }
+        for (int i = head + n_vec * 16 + threadIdx.x; i < first; i += kCompactThreads) cnt += slot_alive[i] != 0;
+    }
+    int before;
+    {
+        int tot;
+        block_excl_scan<kCompactThreads>(cnt, sm, tot);
+        before = tot;
+    }
+
+    const int s = first + threadIdx.x;
+    const int alive = (s < n_slots) && slot_alive[s] != 0;
+    int tot;
+    const int excl = before + block_excl_scan<kCompactThreads>(alive, sm, tot);
+    const int block_end = before + tot;
+
+    if (s < n_slots) {
+        // document of slot s: last d with doc_slot_start[d] <= s (documents without slots are skipped
+        // automatically because their start equals the next document's start)
+        int lo = 0, hi = n_docs;           // invariant: doc_slot_start[lo] <= s < doc_slot_start[hi]
+        while (hi - lo > 1) {
+            int mid = (lo + hi) >> 1;
+            if (doc_slot_start[mid] <= s) lo = mid; else hi = mid;
+        }
+        const int d = lo;
+        const int j = s - doc_slot_start[d];
+        if (j == 0) {
+            // first slot of document d: rows before it; empty documents just before d share the value
+            doc_active_start[d] = excl;
+            for (int e = d - 1; e >= 0 && doc_branch_cnt[e] == 0; --e) doc_active_start[e] = excl;
+        }
+        if (alive) {
+            const int depth = slot_depth[s];
+            const int bs = doc_prefix_len[d] + j * pos_gap;
+            active_slot[excl] = s;
+            doc_id[excl] = d;
+            branch_start[excl] = bs;
+            pos_id[excl] = bs + depth;
+            suffix_off[excl] = s * suffix_cap;
+            suffix_len[excl] = depth;
+        }
+    }
+    if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) {
+        *n_active = block_end;
+        doc_active_start[n_docs] = block_end;
+        for (int e = n_docs - 1; e >= 0 && doc_branch_cnt[e] == 0; --e) doc_active_start[e] = block_end;
+    }
+}
+
+// Split-KV policy.  A work item is (document, chunk of prefix tokens, block of <= 128/G branches).
+// Documents are left whole unless the step has fewer items than SMs; then the largest chunk size
+// 128 * 2^k that yields at least n_sm * Hkv^-1 items is taken, subject to the partial-result and
+// work-list capacities of the workspace.
+constexpr int kCand = 9;             // chunk sizes 128 << 0..7, then "whole document"
+
+__device__ __forceinline__ int chunks_of(int L, int cand) {
+    if (cand == kCand - 1 || L <= 0) return 1;
+    const int S = kTileN << cand;
+    return (L + S - 1) / S;
+}
+
+__global__ void __launch_bounds__(kPlanThreads)
+plan_kernel(int n_docs, int n_slots, int G, int Hkv, int n_sm,
+            const int32_t* __restrict__ doc_prefix_len, const int32_t* __restrict__ doc_active_start,
+            const int32_t* __restrict__ n_active,
+            int32_t* __restrict__ active_slot, int32_t* __restrict__ doc_id, int32_t* __restrict__ branch_start,
+            int32_t* __restrict__ pos_id, int32_t* __restrict__ suffix_off, int32_t* __restrict__ suffix_len,
+            WsHeader* __restrict__ hdr, WorkItem* __restrict__ work, DocSplit* __restrict__ split,
+            int work_cap, int part_cap)
+{
+    if (blockIdx.x > 0) {
+        // tail fill: entries past n_active read -1 in every per-row table
+        const int na = *n_active;
+        for (int i = na + (blockIdx.x - 1) * kPlanThreads + threadIdx.x; i < n_slots; i += (gridDim.x - 1) * kPlanThreads) {
+            active_slot[i] = -1; doc_id[i] = -1; branch_start[i] = -1;
+            pos_id[i] = -1; suffix_off[i] = -1; suffix_len[i] = -1;
+        }
+        return;
+    }
+
+    __shared__ int sm[kPlanThreads / 32 + 1];
+    __shared__ long long red[kCand * 2];
+    __shared__ int s_choice;
+    const int rows_per_block = kTileM / G;
+
+    if (threadIdx.x < kCand * 2) red[threadIdx.x] = 0;
+    __syncthreads();
+    {
+        long long items[kCand], prow[kCand];
+#pragma unroll
+        for (int c = 0; c < kCand; ++c) { items[c] = 0; prow[c] = 0; }
+        for (int d = threadIdx.x; d < n_docs; d += kPlanThreads) {
+            const int rows = doc_active_start[d + 1] - doc_active_start[d];
+            if (rows <= 0) continue;
+            const int mb = (rows + rows_per_block - 1) / rows_per_block;
+            const int L = doc_prefix_len[d];
+#pragma unroll
+            for (int c = 0; c < kCand; ++c) {
+                const int ch = chunks_of(L, c);
+                items[c] += static_cast<long long>(ch) * mb;
+                if (ch > 1) prow[c] += static_cast<long long>(ch) * rows;
+            }
+        }
+#pragma unroll
+        for (int c = 0; c < kCand; ++c) {
+            long long a = items[c], b = prow[c];
+            for (int o = 16; o > 0; o >>= 1) {
+                a += __shfl_down_sync(0xffffffffu, a, o);
+                b += __shfl_down_sync(0xffffffffu, b, o);
+            }
+            if ((threadIdx.x & 31) == 0) {
+                atomicAdd(reinterpret_cast<unsigned long long*>(&red[c]), static_cast<unsigned long long>(a));
+                atomicAdd(reinterpret_cast<unsigned long long*>(&red[kCand + c]), static_cast<unsigned long long>(b));
+            }
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int c = kCand - 1;                              // whole documents
+        while (c > 0 && red[c] * Hkv < n_sm) {
+            const int nc = c - 1;
+            if (red[nc] > work_cap || red[kCand + nc] > part_cap) break;
+            c = nc;
+        }
+        s_choice = c;
+    }
+    __syncthreads();
+    const int cand = s_choice;
+
+    // emit the work list in document order: exclusive scans of items and partial rows per document
+    int run_items = 0, run_part = 0, any_split = 0;
+    for (int base = 0; base < n_docs; base += kPlanThreads) {
+        const int d = base + threadIdx.x;
+        int rows = 0, L = 0, mb = 0, ch = 0;
+        if (d < n_docs) {
+            rows = doc_active_start[d + 1] - doc_active_start[d];
+            L = doc_prefix_len[d];
+            if (rows > 0) {
+                mb = (rows + rows_per_block - 1) / rows_per_block;
+                ch = chunks_of(L, cand);
+            }
+        }
+        const int my_items = ch * mb;
+        const int my_part = ch > 1 ? ch * rows : 0;
+        int tot_i, tot_p;
+        const int ei = run_items + block_excl_scan<kPlanThreads>(my_items, sm, tot_i);
+        const int ep = run_part + block_excl_scan<kPlanThreads>(my_part, sm, tot_p);
+        if (d < n_docs) {
+            split[d].part_base = ch > 1 ? ep : -1;
+            split[d].n_chunks = ch;
+            if (ch > 1) any_split = 1;
+            const int S = (cand == kCand - 1) ? L : (kTileN << cand);
+            int w = ei;
+            for (int c = 0; c < ch; ++c) {
+                const int kb = c * S;
+                const int kc = min(S, L - kb);
+                for (int m = 0; m < mb; ++m, ++w) {
+                    WorkItem it;
+                    it.doc = d;
+                    it.key_begin = kb;
+                    it.key_count = kc > 0 ? kc : 0;
+                    it.row_begin = m * rows_per_block;
+                    it.row_count = min(rows_per_block, rows - it.row_begin);
+                    it.part_base = ch > 1 ? ep + c * rows : -1;
+                    it.with_suffix = (c == ch - 1);
+                    it.pad = 0;
+                    work[w] = it;
+                }
+            }
+        }
+        run_items += tot_i;
+        run_part += tot_p;
+    }
+    const int split_any = __syncthreads_or(any_split);
+    if (threadIdx.x == 0) {
+        hdr->n_work = run_items;
+        hdr->chunk_tokens = (cand == kCand - 1) ? 0 : (kTileN << cand);
+        hdr->n_part_rows = run_part;
+        hdr->any_split = split_any;
+        hdr->ticket = 0;
+        hdr->finished = 0;
+        hdr->work_cap = work_cap;
+        hdr->part_cap = part_cap;
+    }
+}
+
+}  // namespace
+
+WsLayout ws_layout(const hpd_geom& g, int max_docs, int max_slots, int n_sm)
+{
+    WsLayout l{};
+    const int G = g.Hq / g.Hkv;
+    const long long blocks = (static_cast<long long>(max_slots) * G + kTileM - 1) / kTileM;
+    long long work_cap = 2ll * max_docs + 4 * (blocks + 1) + 2ll * n_sm + 64;
+    long long part_cap = 2ll * max_slots + 1024;
+    if (work_cap > 0x7fffffffll) work_cap = 0x7fffffffll;
+    if (part_cap > 0x7fffffffll) part_cap = 0x7fffffffll;
+    l.work_cap = static_cast<int32_t>(work_cap);
+    l.part_cap = static_cast<int32_t>(part_cap);
+    auto up = [](size_t x) { return (x + 255) & ~static_cast<size_t>(255); };
+    size_t off = up(sizeof(WsHeader));
+    l.off_work = off;  off = up(off + sizeof(WorkItem) * static_cast<size_t>(l.work_cap));
+    l.off_split = off; off = up(off + sizeof(DocSplit) * static_cast<size_t>(max_docs > 0 ? max_docs : 1));
+    l.off_ml = off;    off = up(off + sizeof(float) * 2 * static_cast<size_t>(l.part_cap) * g.Hq);
+    l.off_o = off;     off = up(off + sizeof(float) * static_cast<size_t>(l.part_cap) * g.Hq * g.D);
+    l.total = off;
+    return l;
+}
+
+int launch_build_meta(const hpd_geom& g, int n_docs, int n_slots, const int32_t* doc_prefix_len,
+                      const int32_t* doc_branch_cnt, const int32_t* slot_depth, const uint8_t* slot_alive,
+                      int32_t pos_gap, int32_t* doc_kv_start, int32_t* doc_slot_start, int32_t* doc_active_start,
+                      int32_t* active_slot, int32_t* doc_id, int32_t* branch_start, int32_t* pos_id,
+                      int32_t* suffix_off, int32_t* suffix_len, int32_t* n_active, void* workspace,
+                      const WsLayout& lay, int n_sm, int32_t* /*dev_status*/, cudaStream_t stream)
+{
+    char* ws = static_cast<char*>(workspace);
+    WsHeader* hdr = reinterpret_cast<WsHeader*>(ws);
+    WorkItem* work = reinterpret_cast<WorkItem*>(ws + lay.off_work);
+    DocSplit* split = reinterpret_cast<DocSplit*>(ws + lay.off_split);
+
+    doc_scan_kernel<<<1, kScanThreads, 0, stream>>>(n_docs, doc_prefix_len, doc_branch_cnt, doc_kv_start, doc_slot_start);
+    const int cblocks = n_slots > 0 ? (n_slots + kCompactThreads - 1) / kCompactThreads : 1;
+    compact_kernel<<<cblocks, kCompactThreads, 0, stream>>>(
+        n_docs, n_slots, g.suffix_cap, pos_gap, doc_prefix_len, doc_branch_cnt, doc_slot_start, slot_depth, slot_alive,
+        doc_active_start, active_slot, doc_id, branch_start, pos_id, suffix_off, suffix_len, n_active);
+    int fill_blocks = (n_slots + kPlanThreads * 4 - 1) / (kPlanThreads * 4);
+    if (fill_blocks < 1) fill_blocks = 1;
+    if (fill_blocks > 64) fill_blocks = 64;
+    plan_kernel<<<1 + fill_blocks, kPlanThreads, 0, stream>>>(
+        n_docs, n_slots, g.Hq / g.Hkv, g.Hkv, n_sm, doc_prefix_len, doc_active_start, n_active, active_slot, doc_id,
+        branch_start, pos_id, suffix_off, suffix_len, hdr, work, split, lay.work_cap, lay.part_cap);
+    HPD_CUDA_TRY(cudaGetLastError());
+    return HPD_OK;
+}
+
+}  // namespace hpd

@@ -1,0 +1,121 @@
+// hpd_rope and hpd_kv_append: the two streaming kernels around the attention.
+//
+// Both are pure HBM streaming (read + write of the step's new q/k/v rows); one CTA per row,
+// 16-byte accesses, grid sized by max_rows with an early exit on the device-side row count.
+#include "common.cuh"
+
+namespace hpd {
+
+namespace {
+
+constexpr int kRopeThreads = 256;
+
+// One CTA per row.  The row's D/2 (cos, sin) pairs are evaluated once in fp64 (angles reach
+// thousands of radians, where an fp32 product pos * inv_freq already loses ~1e-4 rad), kept in
+// shared memory as fp32, and applied to all Hq + Hkv heads: each thread rotates 8 pairs at a time
+// from one 16-byte load of the low half and one of the high half.
+template <int D>
+__global__ void __launch_bounds__(kRopeThreads)
+rope_kernel(int Hq, int Hkv, double neg_log2_theta_2_over_d, const int32_t* __restrict__ n_active,
+            const int32_t* __restrict__ pos_id, __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ k_new)
+{
+    constexpr int HALF = D / 2;
+    constexpr int CHUNKS = HALF / 8;                 // 16-byte chunks per half
+    __shared__ float cs[HALF], sn[HALF];
+    const int r = blockIdx.x;
+    if (r >= *n_active) return;
+    const int pos = pos_id[r];
+    if (threadIdx.x < HALF) {
+        const double inv_freq = exp2(neg_log2_theta_2_over_d * static_cast<double>(threadIdx.x));
+        double s, c;
+        sincos(static_cast<double>(pos) * inv_freq, &s, &c);
+        cs[threadIdx.x] = static_cast<float>(c);
+        sn[threadIdx.x] = static_cast<float>(s);
+    }
+    __syncthreads();
+    const int items = (Hq + Hkv) * CHUNKS;
+    for (int it = threadIdx.x; it < items; it += kRopeThreads) {
+        const int head = it / CHUNKS, ch = it % CHUNKS;
+        __nv_bfloat16* base = head < Hq ? q + (static_cast<int64_t>(r) * Hq + head) * D
+                                        : k_new + (static_cast<int64_t>(r) * Hkv + (head - Hq)) * D;
+        uint4* plo = reinterpret_cast<uint4*>(base) + ch;
+        uint4* phi = reinterpret_cast<uint4*>(base + HALF) + ch;
+        uint4 lo = *plo, hi = *phi;
+        uint32_t* l = reinterpret_cast<uint32_t*>(&lo);
+        uint32_t* h = reinterpret_cast<uint32_t*>(&hi);
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            const int i = ch * 8 + w * 2;
+            const float a0 = bf16lo(l[w]), a1 = bf16hi(l[w]);
+            const float b0 = bf16lo(h[w]), b1 = bf16hi(h[w]);
+            const float c0 = cs[i], s0 = sn[i], c1 = cs[i + 1], s1 = sn[i + 1];
+            l[w] = pack_bf16(fmaf(a0, c0, -b0 * s0), fmaf(a1, c1, -b1 * s1));
+            h[w] = pack_bf16(fmaf(b0, c0, a0 * s0), fmaf(b1, c1, a1 * s1));
+        }
+        *plo = lo;
+        *phi = hi;
+    }
+}
+
+constexpr int kAppendThreads = 128;
+
+__global__ void __launch_bounds__(kAppendThreads)
+kv_append_kernel(int row_u4 /* Hkv*D*2/16 */, int32_t suffix_cap, int64_t cache_rows,
+                 const int32_t* __restrict__ n_active, const int32_t* __restrict__ suffix_off,
+                 const int32_t* __restrict__ suffix_len,
+                 const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
+                 uint4* __restrict__ suffix_k, uint4* __restrict__ suffix_v, int32_t* __restrict__ dev_status)
+{
+    const int r = blockIdx.x;
+    if (r >= *n_active) return;
+    const int len = suffix_len[r];
+    const int64_t off = suffix_off[r];
+    if (len >= suffix_cap || len < 0) {
+        if (threadIdx.x == 0 && dev_status) atomicOr(dev_status, HPD_S_OVERFLOW);
+        return;
+    }
+    const int64_t dst_row = off + len;
+    if (off < 0 || dst_row >= cache_rows) {
+        if (threadIdx.x == 0 && dev_status) atomicOr(dev_status, HPD_S_BAD_TABLE);
+        return;
+    }
+    const uint4* ks = k_new + static_cast<int64_t>(r) * row_u4;
+    const uint4* vs = v_new + static_cast<int64_t>(r) * row_u4;
+    uint4* kd = suffix_k + dst_row * row_u4;
+    uint4* vd = suffix_v + dst_row * row_u4;
+    for (int i = threadIdx.x; i < row_u4; i += kAppendThreads) {
+        kd[i] = ks[i];
+        vd[i] = vs[i];
+    }
+}
+
+}  // namespace
+
+int launch_rope(const hpd_geom& g, int max_rows, const int32_t* n_active, const int32_t* pos_id,
+                __nv_bfloat16* q, __nv_bfloat16* k_new, cudaStream_t stream)
+{
+    if (max_rows <= 0) return HPD_OK;
+    const double c = -2.0 * log2(static_cast<double>(g.rope_theta)) / static_cast<double>(g.D);
+    if (g.D == 128)
+        rope_kernel<128><<<max_rows, kRopeThreads, 0, stream>>>(g.Hq, g.Hkv, c, n_active, pos_id, q, k_new);
+    else
+        rope_kernel<64><<<max_rows, kRopeThreads, 0, stream>>>(g.Hq, g.Hkv, c, n_active, pos_id, q, k_new);
+    HPD_CUDA_TRY(cudaGetLastError());
+    return HPD_OK;
+}
+
+int launch_kv_append(const hpd_geom& g, int max_rows, int n_slots, const int32_t* n_active, const int32_t* suffix_off,
+                     const int32_t* suffix_len, const __nv_bfloat16* k_new, const __nv_bfloat16* v_new,
+                     __nv_bfloat16* suffix_k, __nv_bfloat16* suffix_v, int32_t* dev_status, cudaStream_t stream)
+{
+    if (max_rows <= 0) return HPD_OK;
+    const int row_u4 = g.Hkv * g.D * 2 / 16;
+    kv_append_kernel<<<max_rows, kAppendThreads, 0, stream>>>(
+        row_u4, g.suffix_cap, static_cast<int64_t>(n_slots) * g.suffix_cap, n_active, suffix_off, suffix_len,
+        reinterpret_cast<const uint4*>(k_new), reinterpret_cast<const uint4*>(v_new),
+        reinterpret_cast<uint4*>(suffix_k), reinterpret_cast<uint4*>(suffix_v), dev_status);
+    HPD_CUDA_TRY(cudaGetLastError());
+    return HPD_OK;
+}
+
+}  // namespace hpd

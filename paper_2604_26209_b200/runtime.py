@@ -1,0 +1,148 @@
+"""Device-side plumbing around the C-ABI calls: upload a synthetic batch and run decode steps.
+
+Holds no arithmetic of the method: tensors are moved to the GPU with PyTorch and every step of
+the path (bookkeeping, rope, append, attention) is a call into ``libhpd.so``.
+"""
+from __future__ import annotations
+
+from typing import Dict, Optional
+
+import numpy as np
+import torch
+
+from . import binding as B
+from .synth import Structure
+
+
+def _bf16(bits: np.ndarray, device) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(device).view(torch.bfloat16)
+
+
+def bits_of(t: torch.Tensor) -> np.ndarray:
+    """bf16 device tensor -> uint16 bit patterns on the host."""
+    return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+class DeviceBatch:
+    """One layer's decode state of a synthetic batch on the GPU."""
+
+    def __init__(self, s: Structure, t: Dict[str, np.ndarray], device="cuda"):
+        self.s, self.g, self.device = s, s.geom, device
+        i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
+        self.doc_prefix_len = i32(s.doc_prefix_len) if s.n_docs else torch.zeros(1, dtype=torch.int32, device=device)
+        self.doc_branch_cnt = i32(s.doc_branch_cnt) if s.n_docs else torch.zeros(1, dtype=torch.int32, device=device)
+        self.slot_depth = i32(s.slot_depth) if s.n_slots else torch.zeros(1, dtype=torch.int32, device=device)
+        self.slot_alive = (torch.from_numpy(np.ascontiguousarray(s.slot_alive, dtype=np.uint8)).to(device)
+                           if s.n_slots else torch.zeros(1, dtype=torch.uint8, device=device))
+        self.prefix_k = _bf16(t["prefix_k"], device) if s.total_prefix else torch.zeros(8, dtype=torch.bfloat16, device=device)
+        self.prefix_v = _bf16(t["prefix_v"], device) if s.total_prefix else torch.zeros(8, dtype=torch.bfloat16, device=device)
+        self.suffix_k = _bf16(t["suffix_k"], device) if s.n_slots else torch.zeros(8, dtype=torch.bfloat16, device=device)
+        self.suffix_v = _bf16(t["suffix_v"], device) if s.n_slots else torch.zeros(8, dtype=torch.bfloat16, device=device)
+        self.meta = B.MetaTables.alloc(self.g, s.n_docs, s.n_slots, s.total_prefix, device)
+        n = max(s.n_slots, 1)
+        self.q = torch.zeros(n, self.g.Hq, self.g.D, dtype=torch.bfloat16, device=device)
+        self.k_new = torch.zeros(n, self.g.Hkv, self.g.D, dtype=torch.bfloat16, device=device)
+        self.v_new = torch.zeros(n, self.g.Hkv, self.g.D, dtype=torch.bfloat16, device=device)
+        self.o = torch.zeros(n, self.g.Hq, self.g.D, dtype=torch.bfloat16, device=device)
+        self.lse = torch.zeros(n, self.g.Hq, dtype=torch.float32, device=device)
+
+    # -- the C-ABI calls, in the order of one step -------------------------------------------
+    def build_meta(self):
+        s = self.s
+        B.hpd_build_meta(self.g, s.n_docs, s.n_slots, self.doc_prefix_len, self.doc_branch_cnt, self.slot_depth,
+                         self.slot_alive, s.pos_gap, self.meta)
+
+    def set_step_inputs(self, q_rows: np.ndarray, k_rows: np.ndarray, v_rows: np.ndarray):
+        """Copy the step's new-token activations (bf16 bits, one row per ACTIVE row) to the device."""
+        n = q_rows.shape[0]
+        if n:
+            self.q[:n].copy_(_bf16(q_rows, self.device))
+            self.k_new[:n].copy_(_bf16(k_rows, self.device))
+            self.v_new[:n].copy_(_bf16(v_rows, self.device))
+
+    def rope(self):
+        B.hpd_rope(self.g, self.s.n_slots, self.meta.n_active, self.meta.pos_id, self.q, self.k_new)
+
+    def kv_append(self):
+        B.hpd_kv_append(self.g, self.s.n_slots, self.s.n_slots, self.meta.n_active, self.meta.suffix_off,
+                        self.meta.suffix_len, self.k_new, self.v_new, self.suffix_k, self.suffix_v, self.meta.dev_status)
+
+    def attn(self, suffix_includes_new=True, lse=True):
+        s = self.s
+        B.hpd_attn_decode(self.g, s.n_docs, s.n_slots, s.n_slots, s.total_prefix, self.q, self.prefix_k, self.prefix_v,
+                          self.suffix_k, self.suffix_v, self.doc_prefix_len, self.meta, suffix_includes_new, self.o,
+                          self.lse if lse else None)
+
+    def step(self, with_meta=True):
+        if with_meta:
+            self.build_meta()
+        self.rope()
+        self.kv_append()
+        self.attn(True)
+
+    # -- read-back --------------------------------------------------------------------------
+    def tables(self) -> Dict[str, np.ndarray]:
+        s = self.s
+        out = {}
+        for name in B.MetaTables.NAMES:
+            a = getattr(self.meta, name).cpu().numpy()
+            n = s.n_docs + 1 if name.startswith("doc_") and name != "doc_id" else s.n_slots
+            out[name] = a[:n].copy()
+        out["n_active"] = int(self.meta.n_active.item())
+        return out
+
+    def status(self) -> int:
+        return int(self.meta.dev_status.item())
+
+
+class DupBatch:
+    """Duplicated-prefix layout for ``std_attn_decode``: every active row gets a private physical copy
+    [its document's prefix ; its cached branch tokens (new token included)].  Built with torch gathers
+    (data preparation for the comparison, not part of the timed path)."""
+
+    def __init__(self, db: DeviceBatch, include_new: bool = True, rows: Optional[int] = None):
+        g, dev = db.g, db.device
+        t = db.tables()
+        n = t["n_active"] if rows is None else min(rows, t["n_active"])
+        self.n = n
+        doc = t["doc_id"][:n].astype(np.int64)
+        L = db.s.doc_prefix_len.astype(np.int64)[doc] if n else np.zeros(0, np.int64)
+        sl = t["suffix_len"][:n].astype(np.int64) + (1 if include_new else 0)
+        sl = np.minimum(sl, g.suffix_cap)
+        lens = L + sl
+        start = np.concatenate([[0], np.cumsum(lens)])[:-1] if n else np.zeros(0, np.int64)
+        total = int(lens.sum())
+        self.max_seq_len = int(lens.max()) if n else 0
+        self.total_tokens = total
+        self.seq_start = torch.from_numpy(start.astype(np.int64)).to(dev) if n else torch.zeros(1, dtype=torch.int64, device=dev)
+        self.seq_len = torch.from_numpy(lens.astype(np.int32)).to(dev) if n else torch.zeros(1, dtype=torch.int32, device=dev)
+        self.n_active = torch.tensor([n], dtype=torch.int32, device=dev)
+        self.dup_k = torch.empty(max(total, 1), g.Hkv, g.D, dtype=torch.bfloat16, device=dev)
+        self.dup_v = torch.empty(max(total, 1), g.Hkv, g.D, dtype=torch.bfloat16, device=dev)
+        kv0 = t["doc_kv_start"].astype(np.int64)
+        soff = t["suffix_off"][:n].astype(np.int64)
+        # chunked gather: index tensors of a few million entries at a time
+        CH = 2048
+        for lo in range(0, n, CH):
+            hi = min(n, lo + CH)
+            src_p, src_s, dst_p, dst_s = [], [], [], []
+            for r in range(lo, hi):
+                src_p.append(np.arange(kv0[doc[r]], kv0[doc[r]] + L[r]))
+                dst_p.append(np.arange(start[r], start[r] + L[r]))
+                src_s.append(np.arange(soff[r], soff[r] + sl[r]))
+                dst_s.append(np.arange(start[r] + L[r], start[r] + lens[r]))
+            for src, dst, K, V in ((src_p, dst_p, db.prefix_k, db.prefix_v), (src_s, dst_s, db.suffix_k, db.suffix_v)):
+                si = torch.from_numpy(np.concatenate(src)).to(dev)
+                di = torch.from_numpy(np.concatenate(dst)).to(dev)
+                if si.numel():
+                    self.dup_k[di] = K.view(-1, g.Hkv, g.D)[si]
+                    self.dup_v[di] = V.view(-1, g.Hkv, g.D)[si]
+        wsb = B.std_workspace_bytes(g, max(n, 1), self.max_seq_len)
+        self.workspace = torch.empty(max(wsb, 16), dtype=torch.uint8, device=dev)
+        self.o = torch.zeros(max(n, 1), g.Hq, g.D, dtype=torch.bfloat16, device=dev)
+        self.lse = torch.zeros(max(n, 1), g.Hq, dtype=torch.float32, device=dev)
+        self.g = g
+
+    def attn(self, q: torch.Tensor):
+        B.std_attn_decode(self.g, self.n, self.max_seq_len, self.n_active, q, self.dup_k, self.dup_v, self.seq_start,
+                          self.seq_len, self.o, self.lse, self.workspace)

@@ -1,0 +1,229 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs.
+
+Bars: integer tables bit-exact; attention outputs max-abs <= 2e-2 and mean-abs <= 2e-3 against the
+oracle; rope within bf16 rounding of the oracle's fp64 rotation; append bit-exact copies.
+"""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2604_26209_b200 import synth
+from tests.util import oracle_step, err_stats, widen
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, MEAN_ABS = 2e-2, 2e-3
+
+
+@pytest.fixture(scope="module")
+def rt():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2604_26209_b200 import runtime
+    return runtime
+
+
+def _ragged(seed, **kw):
+    d = dict(Hq=32, Hkv=8, D=128, theta=500000.0, cap=16, prefix_lens=[300, 0, 129, 1000, 77, 512],
+             branch_cnts=[5, 3, 0, 40, 1, 24], depth_hi=16, seed=seed, alive_frac=0.8)
+    d.update(kw)
+    return synth.config_custom("ragged", **d)
+
+
+STRUCTS = {
+    "tiny": lambda: synth.config_tiny(0),
+    "main_p2": lambda: synth.config_main(n_prompts=2),
+    "ragged": lambda: _ragged(1),
+    "ragged_gap": lambda: _ragged(2, pos_gap=16),
+    "ragged_d64_g2": lambda: _ragged(3, Hq=8, Hkv=4, D=64, theta=10000.0),
+    "ragged_g8": lambda: _ragged(4, Hq=8, Hkv=1),
+    "ragged_g1": lambda: _ragged(5, Hq=4, Hkv=4),
+    "one_group_96": lambda: synth.config_custom("wide", Hq=32, Hkv=8, D=128, theta=500000.0, cap=8,
+                                                prefix_lens=[700], branch_cnts=[96], depth_hi=8, seed=6),
+    "few_alive": lambda: _ragged(7, alive_frac=0.1),
+    "long_small": lambda: synth.config_custom("long", Hq=32, Hkv=8, D=128, theta=500000.0, cap=32,
+                                              prefix_lens=[4096, 1025, 3000], branch_cnts=[12, 12, 12], depth_hi=32, seed=8),
+}
+
+
+def _run_step(rt, s, tb):
+    db = rt.DeviceBatch(s, tb)
+    db.build_meta()
+    tabs = db.tables()
+    act = tabs["active_slot"][: tabs["n_active"]]
+    db.set_step_inputs(tb["q"][act], tb["k_new"][act], tb["v_new"][act])
+    db.rope()
+    db.kv_append()
+    db.attn(True)
+    torch.cuda.synchronize()
+    return db, tabs
+
+
+@pytest.mark.parametrize("name", list(STRUCTS))
+def test_tables_bit_exact(rt, name):
+    s = STRUCTS[name]()
+    tb = synth.make_tensors(s, prefix=False, suffix=False, step=False)
+    from oracle import capi
+    meta = capi.build_meta(s.doc_prefix_len, s.doc_branch_cnt, s.slot_depth, s.slot_alive, s.geom.suffix_cap, s.pos_gap)
+    t2 = dict(prefix_k=np.zeros((max(s.total_prefix, 1), s.geom.Hkv, s.geom.D), np.uint16))
+    t2["prefix_v"] = t2["prefix_k"]
+    t2["suffix_k"] = np.zeros((max(s.n_slots * s.geom.suffix_cap, 1), s.geom.Hkv, s.geom.D), np.uint16)
+    t2["suffix_v"] = t2["suffix_k"]
+    db = rt.DeviceBatch(s, t2)
+    db.build_meta()
+    torch.cuda.synchronize()
+    tabs = db.tables()
+    assert tabs["n_active"] == meta.n_active
+    for nm in capi.Meta.TABLES:
+        assert np.array_equal(tabs[nm], getattr(meta, nm)), nm
+    assert db.status() == 0
+
+
+def test_tables_empty_and_all_retired(rt):
+    from oracle import capi
+    s = _ragged(9, alive_frac=0.0)
+    tb = synth.make_tensors(s)
+    db, tabs = _run_step(rt, s, tb)            # every call must be a no-op with zero rows
+    meta = capi.build_meta(s.doc_prefix_len, s.doc_branch_cnt, s.slot_depth, s.slot_alive, s.geom.suffix_cap, 0)
+    assert tabs["n_active"] == 0
+    for nm in capi.Meta.TABLES:
+        assert np.array_equal(tabs[nm], getattr(meta, nm)), nm
+    assert np.array_equal(rt.bits_of(db.suffix_k), tb["suffix_k"])     # nothing appended
+
+
+@pytest.mark.parametrize("name", list(STRUCTS))
+def test_step_matches_oracle(rt, name):
+    s = STRUCTS[name]()
+    tb = synth.make_tensors(s)
+    meta, want = oracle_step(s, tb)
+    db, tabs = _run_step(rt, s, tb)
+    n = meta.n_active
+    assert tabs["n_active"] == n and db.status() == 0
+
+    # rope: bf16 rounding of the fp64 rotation (|x| <= ~6 -> half-ulp 2^-9 * 4 plus fp32 slack)
+    q_gpu = synth.bf16_bits_to_f32(rt.bits_of(db.q))[:n]
+    k_gpu = synth.bf16_bits_to_f32(rt.bits_of(db.k_new))[:n]
+    for got, ref in ((q_gpu, want.q_rot), (k_gpu, want.k_rot)):
+        tol = np.abs(ref) * (2.0 ** -8 + 1e-5) + 1e-6
+        assert np.all(np.abs(got - ref) <= tol)
+
+    # append: the rotated key and the value land at row off+len, bit-exact copies; nothing else moves
+    sk, sv = rt.bits_of(db.suffix_k), rt.bits_of(db.suffix_v)
+    dst = (meta.suffix_off[:n] + meta.suffix_len[:n]).astype(np.int64)
+    assert np.array_equal(sk[dst], rt.bits_of(db.k_new)[:n])
+    assert np.array_equal(sv[dst], tb["v_new"][meta.active_slot[:n]])
+    untouched = np.ones(sk.shape[0], bool)
+    untouched[dst] = False
+    assert np.array_equal(sk[untouched], tb["suffix_k"][untouched])
+    assert np.array_equal(sv[untouched], tb["suffix_v"][untouched])
+
+    # attention
+    o_gpu = synth.bf16_bits_to_f32(rt.bits_of(db.o))[:n]
+    mx, mean = err_stats(o_gpu, want.o)
+    assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)
+    lse_gpu = db.lse.cpu().numpy()[:n]
+    assert np.max(np.abs(lse_gpu - want.lse)) <= 2e-2
+
+
+@pytest.mark.parametrize("name", ["tiny", "main_p2", "ragged", "ragged_d64_g2", "long_small"])
+def test_std_decode_matches_oracle_and_hpd(rt, name):
+    s = STRUCTS[name]()
+    tb = synth.make_tensors(s)
+    meta, want = oracle_step(s, tb)
+    db, tabs = _run_step(rt, s, tb)
+    n = meta.n_active
+    dup = rt.DupBatch(db, include_new=True)
+    dup.attn(db.q)
+    torch.cuda.synchronize()
+    o_std = synth.bf16_bits_to_f32(rt.bits_of(dup.o))[:n]
+    mx, mean = err_stats(o_std, want.o)
+    assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)
+    o_hpd = synth.bf16_bits_to_f32(rt.bits_of(db.o))[:n]
+    mx, mean = err_stats(o_std, o_hpd)
+    assert mx <= 2 * MAX_ABS and mean <= 2 * MEAN_ABS
+    assert np.max(np.abs(dup.lse.cpu().numpy()[:n] - want.lse)) <= 2e-2
+
+
+def test_std_decode_split_kv_small_batch(rt):
+    """Few rows and long sequences: the split-KV path of the comparison kernel."""
+    s = synth.config_custom("split", Hq=32, Hkv=8, D=128, theta=500000.0, cap=8, prefix_lens=[3000, 2500],
+                            branch_cnts=[2, 1], depth_hi=8, seed=11)
+    tb = synth.make_tensors(s)
+    meta, want = oracle_step(s, tb)
+    db, _ = _run_step(rt, s, tb)
+    dup = rt.DupBatch(db)
+    from paper_2604_26209_b200 import binding
+    assert binding.std_workspace_bytes(s.geom, dup.n, dup.max_seq_len) > 0
+    dup.attn(db.q)
+    torch.cuda.synchronize()
+    mx, mean = err_stats(synth.bf16_bits_to_f32(rt.bits_of(dup.o))[: dup.n], want.o)
+    assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)
+
+
+def test_gpu_output_independent_of_stacking_and_order(rt):
+    """Eq. 4 on the GPU: re-ordering documents / retiring other branches leaves a branch's output
+    within tolerance (the schedule may change the rounding order, not the value)."""
+    s = _ragged(12, alive_frac=1.0)
+    tb = synth.make_tensors(s)
+    db, tabs = _run_step(rt, s, tb)
+    n = tabs["n_active"]
+    base = {int(sl): synth.bf16_bits_to_f32(rt.bits_of(db.o))[r] for r, sl in enumerate(tabs["active_slot"][:n])}
+    alive = s.slot_alive.copy()
+    alive[::3] = 0
+    s2 = replace(s, slot_alive=alive)
+    db2, tabs2 = _run_step(rt, s2, tb)
+    o2 = synth.bf16_bits_to_f32(rt.bits_of(db2.o))
+    for r, sl in enumerate(tabs2["active_slot"][: tabs2["n_active"]]):
+        assert np.max(np.abs(o2[r] - base[int(sl)])) <= MAX_ABS
+
+
+def test_attention_before_append_sees_depth_tokens_only(rt):
+    """suffix_includes_new = 0: the branch sees exactly suffix_len cached tokens (oracle: depth-1 state)."""
+    s = _ragged(13, alive_frac=1.0)
+    s.slot_depth[:] = np.maximum(s.slot_depth, 1)
+    tb = synth.make_tensors(s)
+    # oracle view: the last cached token plays the role of the "new" token of a step at depth-1
+    s_prev = replace(s, slot_depth=s.slot_depth - 1)
+    from oracle import capi
+    meta_prev = capi.build_meta(s_prev.doc_prefix_len, s_prev.doc_branch_cnt, s_prev.slot_depth, s_prev.slot_alive,
+                                s.geom.suffix_cap, 0)
+    f = widen(tb)
+    db = rt.DeviceBatch(s, tb)
+    db.build_meta()
+    tabs = db.tables()
+    n = tabs["n_active"]
+    act = tabs["active_slot"][:n]
+    db.set_step_inputs(tb["q"][act], tb["k_new"][act], tb["v_new"][act])
+    db.rope()
+    db.attn(False)
+    torch.cuda.synchronize()
+    q_rot = synth.bf16_bits_to_f32(rt.bits_of(db.q))[:n]
+    # reference by direct evaluation with the oracle's attention routine on the visible tokens
+    o_gpu = synth.bf16_bits_to_f32(rt.bits_of(db.o))[:n]
+    kv0 = np.concatenate([[0], np.cumsum(s.doc_prefix_len)])
+    for r in range(0, n, 7):
+        d, sl = tabs["doc_id"][r], act[r]
+        K = np.concatenate([f["prefix_k"][kv0[d]:kv0[d + 1]], f["suffix_k"][sl * s.geom.suffix_cap: sl * s.geom.suffix_cap + s.slot_depth[sl]]])
+        V = np.concatenate([f["prefix_v"][kv0[d]:kv0[d + 1]], f["suffix_v"][sl * s.geom.suffix_cap: sl * s.geom.suffix_cap + s.slot_depth[sl]]])
+        o, _ = capi.causal_attention_row(K.shape[0] - 1, q_rot[r], K, V, s.geom.sm_scale)
+        assert np.max(np.abs(o_gpu[r] - o)) <= MAX_ABS
+
+
+def test_overflow_sets_status_and_suppresses_write(rt):
+    s = synth.config_custom("ovf", Hq=4, Hkv=1, D=64, theta=10000.0, cap=4, prefix_lens=[16], branch_cnts=[3],
+                            depth_hi=1, seed=14)
+    s.slot_depth[:] = [0, 4, 2]                 # slot 1 is full
+    tb = synth.make_tensors(s)
+    db = rt.DeviceBatch(s, tb)
+    db.build_meta()
+    db.set_step_inputs(tb["q"], tb["k_new"], tb["v_new"])
+    db.rope()
+    db.kv_append()
+    torch.cuda.synchronize()
+    from paper_2604_26209_b200 import binding
+    assert db.status() & binding.HPD_S_OVERFLOW
+    sk = rt.bits_of(db.suffix_k)
+    assert np.array_equal(sk[4:8], tb["suffix_k"][4:8])          # full slab untouched
+    assert not np.array_equal(sk[0], tb["suffix_k"][0])          # slot 0 got its token
