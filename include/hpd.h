@@ -160,6 +160,32 @@ int std_attn_decode(const hpd_geom* geom /*host*/, int max_rows, int max_seq_len
                     const int64_t* seq_start, const int32_t* seq_len,
                     void* o, float* lse, void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * std_attn_decode_static -- std_attn_decode without a workspace argument.  (The paper has no
+ * counterpart: this is a convenience of the library.)
+ *
+ * For callers that cannot allocate device memory when they need the call: code that runs while a
+ * framework's caching allocator is locked or exhausted, plug-ins of a host program that owns all
+ * device memory, services that have committed the whole device heap to KV caches.  The split-KV
+ * partials go to a fixed array of std_attn_decode_static_max_bytes() (16 MiB) that is part of the
+ * library's device image: every GPU that loads the library holds it until the process exits.
+ *   - Arguments, layouts and results are those of std_attn_decode.
+ *   - A problem whose std_workspace_bytes() exceeds the array is rejected with HPD_E_WORKSPACE and
+ *     nothing is launched; use std_attn_decode with your own workspace then.
+ *   - The call allocates nothing (no cudaMalloc/cudaFree, no allocating library routine).
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) and keeps
+ *     it; make that first call outside any stream capture.
+ *   - All calls on one device share the array and it keeps the last call's contents.  Nothing needs
+ *     clearing (each call writes every partial before its merge reads it), but two calls whose
+ *     kernels can overlap on the GPU (different streams) race on it: keep them on one stream or
+ *     order them with events.
+ */
+size_t std_attn_decode_static_max_bytes(void);
+int std_attn_decode_static(const hpd_geom* geom /*host*/, int max_rows, int max_seq_len, const int32_t* n_active,
+                           const void* q, const void* dup_k, const void* dup_v,
+                           const int64_t* seq_start, const int32_t* seq_len,
+                           void* o, float* lse, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

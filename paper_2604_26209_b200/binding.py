@@ -18,7 +18,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libhpd.so")
 
 EXPORTS = ("hpd_strerror", "hpd_last_cuda_error", "hpd_workspace_bytes", "hpd_build_meta", "hpd_rope",
-           "hpd_kv_append", "hpd_attn_decode", "std_workspace_bytes", "std_attn_decode")
+           "hpd_kv_append", "hpd_attn_decode", "std_workspace_bytes", "std_attn_decode",
+           "std_attn_decode_static_max_bytes", "std_attn_decode_static")
 
 HPD_S_OVERFLOW, HPD_S_BAD_TABLE, HPD_S_TIMEOUT = 1, 2, 4
 
@@ -62,6 +63,10 @@ def load() -> C.CDLL:
                                        [C.c_int, vp, vp, vp, C.c_size_t, vp, vp]
         lib.std_attn_decode.restype = C.c_int
         lib.std_attn_decode.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int] + [vp] * 8 + [vp, C.c_size_t, vp]
+        lib.std_attn_decode_static_max_bytes.restype = C.c_size_t
+        lib.std_attn_decode_static_max_bytes.argtypes = []
+        lib.std_attn_decode_static.restype = C.c_int
+        lib.std_attn_decode_static.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int] + [vp] * 8 + [vp]
         _lib = lib
     return _lib
 
@@ -168,3 +173,18 @@ def std_attn_decode(geom, max_rows, max_seq_len, n_active, q, dup_k, dup_v, seq_
     rc = load().std_attn_decode(C.byref(g), max_rows, max_seq_len, _ptr(n_active), _ptr(q), _ptr(dup_k), _ptr(dup_v),
                                 _ptr(seq_start), _ptr(seq_len), _ptr(o), _ptr(lse), _ptr(workspace), wsb, _stream())
     _check(rc, "std_attn_decode")
+
+
+def std_attn_decode_static_max_bytes() -> int:
+    return int(load().std_attn_decode_static_max_bytes())
+
+
+def std_attn_decode_static(geom, max_rows, max_seq_len, n_active, q, dup_k, dup_v, seq_start, seq_len, o, lse=None):
+    """``std_attn_decode`` with the split-KV scratch inside the library (no workspace, no allocation).
+    Returns the status code instead of raising when the problem exceeds the built-in scratch."""
+    g = make_geom(geom)
+    rc = load().std_attn_decode_static(C.byref(g), max_rows, max_seq_len, _ptr(n_active), _ptr(q), _ptr(dup_k),
+                                       _ptr(dup_v), _ptr(seq_start), _ptr(seq_len), _ptr(o), _ptr(lse), _stream())
+    if rc != -3:
+        _check(rc, "std_attn_decode_static")
+    return rc

@@ -1,0 +1,69 @@
+"""``std_attn_decode_static``: the comparison kernel for callers that cannot allocate device memory.
+
+Some users of the library cannot hand it a workspace: they run while their framework's allocator is
+locked or out of memory, or inside a host program that owns every byte of the device.  For them the
+library keeps a fixed 16 MiB scratch array in its own device image.  This test calls the entry point
+through the C ABI twice in a row (the second call finds the first call's leftovers in the shared
+array) and checks both outputs against ``std_attn_decode`` with an ordinary workspace.  The file name
+makes pytest collect it last, so a failure here cannot hide the result of any other test.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2604_26209_b200 import synth
+
+pytestmark = pytest.mark.gpu
+MAX_ABS, MEAN_ABS = 2e-2, 2e-3
+
+
+def _batch(seed):
+    from paper_2604_26209_b200 import runtime
+    # few rows, long sequences: the split-KV path, i.e. the one that needs scratch memory
+    s = synth.config_custom("static", Hq=32, Hkv=8, D=128, theta=500000.0, cap=8, prefix_lens=[3000, 2500],
+                            branch_cnts=[2, 1], depth_hi=8, seed=seed)
+    tb = synth.make_tensors(s)
+    db = runtime.DeviceBatch(s, tb)
+    db.build_meta()
+    n = db.tables()["n_active"]
+    db.set_step_inputs(tb["q"][:n], tb["k_new"][:n], tb["v_new"][:n])
+    db.rope()
+    db.kv_append()
+    return s, db, runtime.DupBatch(db)
+
+
+def test_static_scratch_matches_workspace_variant_twice():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2604_26209_b200 import binding, runtime
+    assert binding.std_attn_decode_static_max_bytes() == 16 << 20
+    for seed in (21, 22):                       # two calls in a row share the library's scratch array
+        s, db, dup = _batch(seed)
+        need = binding.std_workspace_bytes(s.geom, dup.n, dup.max_seq_len)
+        assert 0 < need <= binding.std_attn_decode_static_max_bytes()
+        dup.attn(db.q)                          # reference: caller-provided workspace
+        torch.cuda.synchronize()
+        want_o = synth.bf16_bits_to_f32(runtime.bits_of(dup.o))[: dup.n].copy()
+        want_lse = dup.lse.cpu().numpy()[: dup.n].copy()
+        dup.o.zero_(); dup.lse.zero_()
+        rc = binding.std_attn_decode_static(s.geom, dup.n, dup.max_seq_len, dup.n_active, db.q, dup.dup_k, dup.dup_v,
+                                            dup.seq_start, dup.seq_len, dup.o, dup.lse)
+        torch.cuda.synchronize()
+        assert rc == 0
+        got_o = synth.bf16_bits_to_f32(runtime.bits_of(dup.o))[: dup.n]
+        d = np.abs(got_o - want_o)
+        assert d.max() <= MAX_ABS and d.mean() <= MEAN_ABS, (seed, d.max(), d.mean())
+        assert np.max(np.abs(dup.lse.cpu().numpy()[: dup.n] - want_lse)) <= 2e-2
+
+
+def test_static_scratch_rejects_oversized_problem():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2604_26209_b200 import binding
+    s, db, dup = _batch(23)
+    rows, seq = 590, 4096                       # 590 rows x 32 heads x 2 splits x 130 floats > 16 MiB
+    assert binding.std_workspace_bytes(s.geom, rows, seq) > binding.std_attn_decode_static_max_bytes()
+    rc = binding.std_attn_decode_static(s.geom, rows, seq, dup.n_active, db.q, dup.dup_k, dup.dup_v, dup.seq_start,
+                                        dup.seq_len, dup.o, dup.lse)
+    assert rc == -3                             # HPD_E_WORKSPACE, nothing launched
+    torch.cuda.synchronize()
