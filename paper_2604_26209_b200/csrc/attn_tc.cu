@@ -3,14 +3,20 @@
 // One persistent CTA per SM walks the step's work units.  A unit = (work item, kv head): up to
 // 128/G branches of one document (rows = branches x G query heads, the M dimension) against a chunk
 // of that document's prefix, so each prefix K/V byte is read from HBM once for all of the document's
-// branches.  The branches' own cached tokens ("suffix") are gathered into further K/V tiles of the
-// same pipeline and masked block-diagonally (a row sees only its own branch's columns).
+// branches.  Keys are consumed in tiles of 64: first the prefix tiles, then tiles into which the
+// branches' own cached tokens ("suffix") are packed back to back by TMA boxes of 1..16 cache rows;
+// those tiles are masked block-diagonally (a row sees only its own branch's columns).  Even tiles
+// form stream A, odd tiles stream B, each with its own MMA-issuing warp, softmax group, score
+// buffer, probability tile and output accumulator, so the two streams run as independent
+// online-softmax pipelines over one K/V stream (a split-KV inside the CTA); the epilogue merges them.
 //
-//   warp 0      TMA producer: Q tile, prefix K tiles, prefix V tiles (128B-swizzled boxes)
-//   warp 1      MMA issuer:   S = Q K^T  (tcgen05.mma, accumulators in TMEM), O += P V
-//   warps 2-5   softmax:      one thread per row; S from TMEM, online max/sum, P (bf16) to shared
-//                             memory, rare rescale of O in TMEM, epilogue
-//   warps 6-9   gather:       branch-cache rows -> swizzled K/V tiles with cp.async
+//   warp 0        TMA producer: Q tile (double buffered), prefix K/V tiles (lane 0), suffix boxes (all lanes)
+//   warps 1-2     MMA issuers of streams A and B: S = Q K^T and O += P V (tcgen05.mma, TMEM accumulators)
+//   warp 3        idle (it completes the first warpgroup, which gives its registers away)
+//   warps 4-7     softmax A     one thread per row: S from TMEM, online max/sum, P (bf16) to shared
+//   warps 8-11    softmax B     memory, rare rescale of O in TMEM; both groups share the epilogue
+//
+// TMEM columns: S_A [0,64)  S_B [64,128)  O_A [128,256)  O_B [256,384).
 //
 // All waits are bounded: a wait that gives up raises HPD_S_TIMEOUT in the status word and the CTA
 // drains and exits (TMEM is released on every path).
@@ -25,38 +31,51 @@ namespace hpd {
 
 namespace {
 
-constexpr int kThreads = 320;
-constexpr int kTile = 128;                 // rows and keys per tile
-constexpr int kHalfBytes = kTile * 128;    // one 64-element half of a tile: 128 rows x 128 B
-constexpr int kPBytes = 2 * kHalfBytes;    // P tile: 128 rows x 128 keys bf16
+constexpr int kWarps = 12;
+constexpr int kThreads = kWarps * 32;
+constexpr int kM = 128;                    // rows of a tile
+constexpr int kN = 64;                     // keys of a tile
+constexpr int kQHalf = kM * 128;           // one 64-element half of the Q tile: 128 rows x 128 B
+constexpr int kKHalf = kN * 128;           // one 64-element half of a K or V tile: 64 keys x 128 B
+constexpr int kPBytes = kM * 128;          // P tile: 128 rows x 64 keys bf16
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleSlack = 8.0f;      // tolerated growth of the row maximum (log2 units) before O is rescaled
 constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz
+constexpr uint32_t kColS = 0, kColO = 128;
+// registers per thread after the warpgroups have traded them (3 x 128 threads, 168 each at launch)
+constexpr int kRegsIo = 80, kRegsSoftmax = 208;
+constexpr int kBoxKinds = 5;               // suffix boxes of 1, 2, 4, 8, 16 cache rows
+constexpr int kRounds = 4;                 // a unit has at most 128 branches: 4 rounds of 32 lanes
 
 template <int D> struct Cfg {
     static constexpr int HALVES = D / 64;
-    static constexpr int TILE_BYTES = HALVES * kHalfBytes;     // Q, K or V tile
-    static constexpr int NK = D == 128 ? 3 : 4;                 // K stages
-    static constexpr int NV = D == 128 ? 2 : 4;                 // V stages
+    static constexpr int Q_BYTES = HALVES * kQHalf;
+    static constexpr int KV_BYTES = HALVES * kKHalf;            // one K or V tile
+    static constexpr int NK = D == 128 ? 4 : 8;                  // K stages
+    static constexpr int NV = D == 128 ? 4 : 8;                  // V stages
     static constexpr int OFF_Q = 0;
-    static constexpr int OFF_K = OFF_Q + TILE_BYTES;
-    static constexpr int OFF_V = OFF_K + NK * TILE_BYTES;
-    static constexpr int OFF_P = OFF_V + NV * TILE_BYTES;
-    static constexpr int OFF_MISC = OFF_P + kPBytes;
-    static constexpr int SMEM = OFF_MISC + 2048 + 1024;         // + misc + slack for 1024-B alignment
+    static constexpr int OFF_P = OFF_Q + 2 * Q_BYTES;
+    static constexpr int OFF_K = OFF_P + 2 * kPBytes;
+    static constexpr int OFF_V = OFF_K + NK * KV_BYTES;
+    static constexpr int OFF_MISC = OFF_V + NV * KV_BYTES;
+    static constexpr int SMEM = OFF_MISC + 2048 + 1024;          // + misc + slack for 1024-B alignment
 };
+static_assert(Cfg<128>::SMEM <= 232448, "shared memory budget");
 
 struct Misc {
-    unsigned long long q_full, q_empty, p_full, p_empty;
-    unsigned long long k_full[4], k_empty[4], v_full[4], v_empty[4];
-    unsigned long long s_full[2], s_empty[2];
+    unsigned long long q_full[2], q_empty[2];
+    unsigned long long k_full[8], k_empty[8], v_full[8], v_empty[8];
+    unsigned long long s_full[2], s_empty[2], p_full[2], p_empty[2], o_full[2];
+    unsigned long long o_free, ml_full;
     uint32_t tmem_base;
     int abort_flag;
-    int wt[2][4];
-    int cs[2][kTile + 4];
 };
 static_assert(sizeof(Misc) <= 2048, "misc block");
+
+struct SufMaps {                            // tensor maps of the branch cache, one per box height
+    CUtensorMap k[kBoxKinds], v[kBoxKinds];
+};
 
 struct TcParams {
     AttnArgs a;
@@ -153,95 +172,95 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void named_bar(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
-// barrier over a 128-thread role group that also AND-reduces a flag, so that exits stay uniform
-__device__ __forceinline__ bool named_bar_and(int id, bool v) {
-    uint32_t r;
-    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred p, %2, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(r) : "r"(v ? 1u : 0u), "r"(id) : "memory");
-    return r != 0;
-}
+template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
 // Shared-memory matrix descriptors (128-byte swizzle; version field = 1).
 //   K-major  (Q, K, P): rows of 128 B; groups of 8 rows 1024 B apart (SBO); LBO unused.
 //   MN-major (V):       rows (keys) of 128 B holding 64 head-dim elements; 8-key groups 1024 B apart
-//                       (SBO); the next 64 head-dim elements 16 KiB further (LBO).
+//                       (SBO); the next 64 head-dim elements one tile half further (LBO).
 __device__ __forceinline__ uint64_t desc_kmajor(uint32_t saddr) {
     return static_cast<uint64_t>((saddr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
 }
 __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr) {
-    return static_cast<uint64_t>((saddr >> 4) & 0x3FFF) | (static_cast<uint64_t>(kHalfBytes >> 4) << 16) | (64ull << 32) |
+    return static_cast<uint64_t>((saddr >> 4) & 0x3FFF) | (static_cast<uint64_t>(kKHalf >> 4) << 16) | (64ull << 32) |
            (1ull << 46) | (2ull << 61);
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N given; B either K-major (Q K^T) or MN-major (P V).
 __device__ __forceinline__ uint32_t make_idesc(int N, int b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(b_mn_major) << 16) |
-           (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(kTile >> 4) << 24);
+           (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(kM >> 4) << 24);
 }
 
 // ------------------------------------------------------------------------------------------------
 // per-unit bookkeeping shared by all roles (every role recomputes it from the same global data)
 // ------------------------------------------------------------------------------------------------
 struct Unit {
-    int doc, head, key_count, part_base, row_begin, nb /*branches*/, with_suffix;
+    int head, key_count, part_base, row_begin, nb /*branches*/, with_suffix;
     int row0;        // first global row
     int kv_row0;     // first global prefix token row
     int np;          // prefix tiles
 };
 
-__device__ __forceinline__ Unit load_unit(const TcParams& p, int w) {
+__device__ __forceinline__ Unit load_unit(const TcParams& p, int w, int n_units) {
+    Unit u{};
+    if (w >= n_units) return u;
     const int Hkv = p.a.g.Hkv;
     const WorkItem it = p.work[w / Hkv];
-    Unit u;
-    u.doc = it.doc; u.head = w % Hkv; u.key_count = it.key_count; u.part_base = it.part_base;
+    u.head = w % Hkv; u.key_count = it.key_count; u.part_base = it.part_base;
     u.row_begin = it.row_begin; u.nb = it.row_count; u.with_suffix = it.with_suffix;
     u.row0 = p.a.doc_active_start[it.doc] + it.row_begin;
     u.kv_row0 = p.a.doc_kv_start[it.doc] + it.key_begin;
-    u.np = (it.key_count + kTile - 1) / kTile;
+    u.np = (it.key_count + kN - 1) / kN;
     return u;
 }
 
-__device__ __forceinline__ int branch_suffix_len(const TcParams& p, int row) {
-    int n = p.a.suffix_len[row] + p.a.suffix_extra;
-    n = n < 0 ? 0 : n;
-    return n > p.a.g.suffix_cap ? p.a.g.suffix_cap : n;
-}
+// Branch-cache table of a unit, spread over the lanes of a warp: entry r of lane i belongs to branch
+// i + 32 r.  len = cached tokens visible to the branch (0 for a bad table entry), off = first cache row.
+struct SufTab {
+    int len[kRounds], off[kRounds];
+    int bad;
+};
 
-// total cached tokens of the unit's branches (whole warp calls it)
-__device__ __forceinline__ int suffix_total_warp(const TcParams& p, const Unit& u, int lane) {
-    if (!u.with_suffix) return 0;
-    int s = 0;
-    for (int b = lane; b < u.nb; b += 32) s += branch_suffix_len(p, u.row0 + b);
+__device__ __forceinline__ SufTab load_suftab(const TcParams& p, const Unit& u, int lane) {
+    SufTab t;
+    t.bad = 0;
+    const int64_t cache_rows = static_cast<int64_t>(p.a.n_slots) * p.a.g.suffix_cap;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    return s;
-}
-
-// exclusive scan of the branches' cached lengths over a 128-thread role group -> cs[0..128]; returns total
-__device__ __forceinline__ int suffix_scan_group(const TcParams& p, const Unit& u, Misc* misc, int which, int t /*0..127*/, int bar_id) {
-    int* cs = misc->cs[which];
-    int* wt = misc->wt[which];
-    int len = 0;
-    if (u.with_suffix && t < u.nb) len = branch_suffix_len(p, u.row0 + t);
-    int incl = len;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        int v = __shfl_up_sync(0xffffffffu, incl, o);
-        if ((t & 31) >= o) incl += v;
+    for (int r = 0; r < kRounds; ++r) {
+        t.len[r] = 0; t.off[r] = 0;
+        const int b = lane + 32 * r;
+        if (u.with_suffix && b < u.nb) {
+            const int row = u.row0 + b;
+            int n = p.a.suffix_len[row] + p.a.suffix_extra;
+            n = n < 0 ? 0 : (n > p.a.g.suffix_cap ? p.a.g.suffix_cap : n);
+            const int64_t srow = p.a.suffix_off[row];
+            if (srow < 0 || srow + n > cache_rows) t.bad = 1;
+            else { t.len[r] = n; t.off[r] = static_cast<int>(srow); }
+        }
     }
-    named_bar(bar_id);                       // previous unit's readers are done with cs/wt
-    if ((t & 31) == 31) wt[t >> 5] = incl;
-    named_bar(bar_id);
-    int off = 0;
-    for (int w = 0; w < (t >> 5); ++w) off += wt[w];
-    const int total = wt[0] + wt[1] + wt[2] + wt[3];
-    cs[t] = off + incl - len;
-    if (t == kTile - 1) cs[kTile] = total;
-    named_bar(bar_id);
-    return total;
+    return t;
+}
+
+// exclusive scan of the lengths over the unit's branches (packed column of each branch's first token); returns the total
+__device__ __forceinline__ int scan_suftab(const SufTab& t, int lane, int* cs /*[kRounds]*/) {
+    int carry = 0;
+#pragma unroll
+    for (int r = 0; r < kRounds; ++r) {
+        int incl = t.len[r];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        cs[r] = carry + incl - t.len[r];
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    return carry;
+}
+
+__device__ __forceinline__ int tile_cols(const Unit& u, int stot, int j) {
+    return j < u.np ? min(kN, u.key_count - j * kN) : min(kN, stot - (j - u.np) * kN);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -250,7 +269,7 @@ __device__ __forceinline__ int suffix_scan_group(const TcParams& p, const Unit& 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                   const __grid_constant__ CUtensorMap map_v, const TcParams p)
+                   const __grid_constant__ CUtensorMap map_v, const __grid_constant__ SufMaps smaps, const TcParams p)
 {
     using C = Cfg<D>;
     extern __shared__ uint8_t smem_raw[];
@@ -259,19 +278,27 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = p.G;
     const int n_units = p.hdr->n_work * p.a.g.Hkv;
+    const int stride = gridDim.x;
 
     if (threadIdx.x == 0) {
-        mbar_init(&misc->q_full, 1);  mbar_init(&misc->q_empty, 1);
-        mbar_init(&misc->p_full, 4);  mbar_init(&misc->p_empty, 1);
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&misc->q_full[i], 1);  mbar_init(&misc->q_empty[i], 2);
+            mbar_init(&misc->s_full[i], 1);  mbar_init(&misc->s_empty[i], 4);
+            mbar_init(&misc->p_full[i], 4);  mbar_init(&misc->p_empty[i], 1);
+            mbar_init(&misc->o_full[i], 1);
+        }
+        for (int i = 0; i < 8; ++i) {
             mbar_init(&misc->k_full[i], 1); mbar_init(&misc->k_empty[i], 1);
             mbar_init(&misc->v_full[i], 1); mbar_init(&misc->v_empty[i], 1);
         }
-        for (int i = 0; i < 2; ++i) { mbar_init(&misc->s_full[i], 1); mbar_init(&misc->s_empty[i], 4); }
+        mbar_init(&misc->o_free, 8); mbar_init(&misc->ml_full, 8);
         misc->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        fence_async_smem();
     }
+    // stale tile contents are multiplied by zero probabilities: they must be finite from the start
+    for (int i = threadIdx.x; i < (C::OFF_MISC - C::OFF_K) / 16; i += kThreads)
+        reinterpret_cast<uint4*>(smem + C::OFF_K)[i] = make_uint4(0, 0, 0, 0);
+    fence_async_smem();
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&misc->tmem_base)), "r"(512) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -280,189 +307,252 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&misc->tmem_base);
-    const uint32_t tmem_o = tmem + 2 * kTile;            // columns [256, 256 + D)
 
     if (warp == 0) {
         // ======================================= TMA producer =======================================
-        uint32_t qi = 0, kc = 0, vc = 0;
+        reg_dealloc<kRegsIo>();
+        uint32_t qc = 0, kc = 0, vc = 0;
         bool ok = true;
-        for (int w = blockIdx.x; w < n_units && ok; w += gridDim.x) {
-            const Unit u = load_unit(p, w);
-            const int stot = suffix_total_warp(p, u, lane);
-            const int ns = (stot + kTile - 1) / kTile;
-            if (u.np + ns == 0) continue;
-            if (lane == 0) {
-                ok = mbar_wait(&misc->q_empty, (qi & 1) ^ 1, misc);
-                if (ok) {
-                    mbar_expect_tx(&misc->q_full, C::TILE_BYTES);
+        Unit u = load_unit(p, blockIdx.x, n_units);
+        SufTab tab = load_suftab(p, u, lane);
+        for (int w = blockIdx.x; w < n_units && ok; w += stride) {
+            const Unit nxt = load_unit(p, w + stride, n_units);
+            const SufTab ntab = load_suftab(p, nxt, lane);
+            int cs[kRounds];
+            const int stot = scan_suftab(tab, lane, cs);
+            if (__any_sync(0xffffffffu, tab.bad) && lane == 0 && p.a.dev_status) atomicOr(p.a.dev_status, HPD_S_BAD_TABLE);
+            const int nt = u.np + (stot + kN - 1) / kN;
+            if (nt > 0) {
+                const int qb = qc & 1;
+                ok = mbar_wait_warp(&misc->q_empty[qb], ((qc >> 1) & 1) ^ 1, misc);
+                if (!ok) break;
+                if (lane == 0) {
+                    mbar_expect_tx(&misc->q_full[qb], C::Q_BYTES);
                     for (int h = 0; h < C::HALVES; ++h)
-                        tma_load_4d(smem + C::OFF_Q + h * kHalfBytes, &map_q, &misc->q_full, h * 64, 0, u.head, u.row0);
+                        tma_load_4d(smem + C::OFF_Q + qb * C::Q_BYTES + h * kQHalf, &map_q, &misc->q_full[qb], h * 64, 0, u.head, u.row0);
                 }
-                // Every ring slot is waited for in order, also the suffix tiles' slots that the gather warps
-                // fill: a waiter that skipped slots could otherwise test an mbarrier phase two behind.
-                for (int t = 0; t < u.np + ns && ok; ++t) {
-                    const int ks = kc % C::NK, vs = vc % C::NV;
-                    ok = mbar_wait(&misc->k_empty[ks], ((kc / C::NK) & 1) ^ 1, misc);
-                    if (!ok) break;
+                ++qc;
+                // One tile: a prefix tile is two boxes issued by lane 0; a suffix tile is packed from boxes of
+                // 1..16 cache rows, every lane placing the part of its branches that falls into the tile.
+                auto fill = [&](int t, uint8_t* tile, unsigned long long* full, const CUtensorMap& pre, const CUtensorMap* suf) {
                     if (t < u.np) {
-                        mbar_expect_tx(&misc->k_full[ks], C::TILE_BYTES);
-                        for (int h = 0; h < C::HALVES; ++h)
-                            tma_load_3d(smem + C::OFF_K + ks * C::TILE_BYTES + h * kHalfBytes, &map_k, &misc->k_full[ks],
-                                        h * 64, u.head, u.kv_row0 + t * kTile);
-                    }
-                    ok = mbar_wait(&misc->v_empty[vs], ((vc / C::NV) & 1) ^ 1, misc);
-                    if (!ok) break;
-                    if (t < u.np) {
-                        mbar_expect_tx(&misc->v_full[vs], C::TILE_BYTES);
-                        for (int h = 0; h < C::HALVES; ++h)
-                            tma_load_3d(smem + C::OFF_V + vs * C::TILE_BYTES + h * kHalfBytes, &map_v, &misc->v_full[vs],
-                                        h * 64, u.head, u.kv_row0 + t * kTile);
-                    }
-                    ++kc; ++vc;
-                }
-            }
-            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-            kc = __shfl_sync(0xffffffffu, kc, 0);
-            vc = __shfl_sync(0xffffffffu, vc, 0);
-            ++qi;
-        }
-    } else if (warp == 1) {
-        // ======================================== MMA issuer ========================================
-        uint32_t qi = 0, kc = 0, vc = 0, sc = 0, pc = 0;
-        bool ok = true;
-        const uint32_t q_addr = smem_u32(smem + C::OFF_Q), p_addr = smem_u32(smem + C::OFF_P);
-        for (int w = blockIdx.x; w < n_units && ok; w += gridDim.x) {
-            const Unit u = load_unit(p, w);
-            const int stot = suffix_total_warp(p, u, lane);
-            const int ns = (stot + kTile - 1) / kTile;
-            const int nt = u.np + ns;
-            if (nt == 0) continue;
-            if (lane == 0) {
-                ok = mbar_wait(&misc->q_full, qi & 1, misc);
-                auto tile_cols = [&](int j) {
-                    return j < u.np ? min(kTile, u.key_count - j * kTile) : min(kTile, stot - (j - u.np) * kTile);
-                };
-                auto issue_qk = [&](int j) {
-                    const int ks = kc % C::NK, sb = sc & 1;
-                    if (!mbar_wait(&misc->k_full[ks], (kc / C::NK) & 1, misc)) return false;
-                    if (!mbar_wait(&misc->s_empty[sb], ((sc >> 1) & 1) ^ 1, misc)) return false;
-                    tc_fence_after();
-                    const int n_pad = (tile_cols(j) + 15) & ~15;
-                    const uint32_t idesc = make_idesc(n_pad, 0);
-                    const uint32_t k_addr = smem_u32(smem + C::OFF_K + ks * C::TILE_BYTES);
+                        if (lane == 0) {
+                            mbar_expect_tx(full, C::KV_BYTES);
+                            for (int h = 0; h < C::HALVES; ++h)
+                                tma_load_3d(tile + h * kKHalf, &pre, full, h * 64, u.head, u.kv_row0 + t * kN);
+                        }
+                    } else {
+                        const int c_lo = (t - u.np) * kN, c_hi = min(stot, c_lo + kN);
+                        if (lane == 0) mbar_expect_tx(full, static_cast<uint32_t>(c_hi - c_lo) * D * 2);
 #pragma unroll
-                    for (int k = 0; k < D / 16; ++k) {
-                        const uint32_t off = (k >> 2) * kHalfBytes + (k & 3) * 32;
-                        tc_mma(tmem + sb * kTile, desc_kmajor(q_addr + off), desc_kmajor(k_addr + off), idesc, k > 0);
+                        for (int r = 0; r < kRounds; ++r) {
+                            const int lo = max(cs[r], c_lo), hi = min(cs[r] + tab.len[r], c_hi);
+                            int n = hi - lo;
+                            int row = tab.off[r] + (lo - cs[r]);
+                            int col = lo - c_lo;
+                            while (n > 0) {
+                                const int kind = min(kBoxKinds - 1, 31 - __clz(n));
+                                for (int h = 0; h < C::HALVES; ++h)
+                                    tma_load_3d(tile + h * kKHalf + col * 128, &suf[kind], full, h * 64, u.head, row);
+                                row += 1 << kind; col += 1 << kind; n -= 1 << kind;
+                            }
+                        }
                     }
-                    tc_commit(&misc->k_empty[ks]);
-                    tc_commit(&misc->s_full[sb]);
-                    if (j == nt - 1) tc_commit(&misc->q_empty);
-                    ++kc; ++sc;
-                    return true;
                 };
-                if (ok) ok = issue_qk(0);
-                for (int j = 0; j < nt && ok; ++j) {
-                    if (j + 1 < nt) { ok = issue_qk(j + 1); if (!ok) break; }
-                    const int vs = vc % C::NV;
-                    ok = mbar_wait(&misc->p_full, pc & 1, misc);
-                    if (!ok) break;
-                    ok = mbar_wait(&misc->v_full[vs], (vc / C::NV) & 1, misc);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t idesc = make_idesc(D, 1);
-                    const uint32_t v_addr = smem_u32(smem + C::OFF_V + vs * C::TILE_BYTES);
-                    const int nk = (tile_cols(j) + 15) >> 4;
-                    for (int k = 0; k < nk; ++k) {
-                        const uint32_t a_off = (k >> 2) * kHalfBytes + (k & 3) * 32;
-                        tc_mma(tmem_o, desc_kmajor(p_addr + a_off), desc_mnmajor(v_addr + k * 2048), idesc, (j > 0 || k > 0));
+                // K runs two tiles ahead of V, the order in which the MMA warps consume them
+                for (int t = 0; t < nt + 2 && ok; ++t) {
+                    if (t < nt) {
+                        const int ks = kc % C::NK;
+                        ok = mbar_wait_warp(&misc->k_empty[ks], ((kc / C::NK) & 1) ^ 1, misc);
+                        if (!ok) break;
+                        fill(t, smem + C::OFF_K + ks * C::KV_BYTES, &misc->k_full[ks], map_k, smaps.k);
+                        ++kc;
                     }
-                    tc_commit(&misc->v_empty[vs]);
-                    tc_commit(&misc->p_empty);
-                    ++vc; ++pc;
+                    if (t >= 2) {
+                        const int vs = vc % C::NV;
+                        ok = mbar_wait_warp(&misc->v_empty[vs], ((vc / C::NV) & 1) ^ 1, misc);
+                        if (!ok) break;
+                        fill(t - 2, smem + C::OFF_V + vs * C::KV_BYTES, &misc->v_full[vs], map_v, smaps.v);
+                        ++vc;
+                    }
+                    __syncwarp();
                 }
             }
-            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-            kc = __shfl_sync(0xffffffffu, kc, 0); vc = __shfl_sync(0xffffffffu, vc, 0);
-            sc = __shfl_sync(0xffffffffu, sc, 0); pc = __shfl_sync(0xffffffffu, pc, 0);
-            ++qi;
+            u = nxt;
+            tab = ntab;
         }
-    } else if (warp < 6) {
-        // ========================================= softmax ==========================================
+    } else if (warp < 3) {
+        // ================================ MMA issuers (one per stream) ===============================
+        reg_dealloc<kRegsIo>();
+        const int x = warp - 1;                          // stream: tiles x, x+2, ...
+        uint32_t qc = 0, tiles = 0, unit_idx = 0;         // units with tiles so far; tiles of earlier units
+        uint32_t sc = 0, pc = 0;                          // this stream: S tiles issued, P tiles consumed
+        bool ok = true;
+        const uint32_t p_addr = smem_u32(smem + C::OFF_P + x * kPBytes);
+        const uint32_t tmem_s = tmem + kColS + x * kN, tmem_o = tmem + kColO + x * 128;
+        Unit u = load_unit(p, blockIdx.x, n_units);
+        SufTab tab = load_suftab(p, u, lane);
+        for (int w = blockIdx.x; w < n_units && ok; w += stride, ++unit_idx) {
+            const Unit nxt = load_unit(p, w + stride, n_units);
+            const SufTab ntab = load_suftab(p, nxt, lane);
+            int cs[kRounds];
+            const int stot = scan_suftab(tab, lane, cs);
+            const int nt = u.np + (stot + kN - 1) / kN;
+            if (nt > 0) {
+                const int qb = qc & 1;
+                ++qc;
+                if (lane == 0) {
+                    const uint32_t q_addr = smem_u32(smem + C::OFF_Q + qb * C::Q_BYTES);
+                    ok = mbar_wait(&misc->q_full[qb], ((qc - 1) >> 1) & 1, misc);
+                    auto issue_qk = [&](int j) {
+                        const uint32_t kt = tiles + j;
+                        const int ks = kt % C::NK;
+                        if (!mbar_wait(&misc->k_full[ks], (kt / C::NK) & 1, misc)) return false;
+                        if (!mbar_wait(&misc->s_empty[x], (sc & 1) ^ 1, misc)) return false;
+                        tc_fence_after();
+                        const int n_pad = (tile_cols(u, stot, j) + 15) & ~15;
+                        const uint32_t idesc = make_idesc(n_pad, 0);
+                        const uint32_t k_addr = smem_u32(smem + C::OFF_K + ks * C::KV_BYTES);
+#pragma unroll
+                        for (int k = 0; k < D / 16; ++k) {
+                            const uint32_t qoff = (k >> 2) * kQHalf + (k & 3) * 32;
+                            const uint32_t koff = (k >> 2) * kKHalf + (k & 3) * 32;
+                            tc_mma(tmem_s, desc_kmajor(q_addr + qoff), desc_kmajor(k_addr + koff), idesc, k > 0);
+                        }
+                        tc_commit(&misc->k_empty[ks]);
+                        tc_commit(&misc->s_full[x]);
+                        if (j + 2 >= nt) tc_commit(&misc->q_empty[qb]);     // this stream's last use of the Q tile
+                        ++sc;
+                        return true;
+                    };
+                    if (x >= nt) {
+                        if (ok) mbar_arrive(&misc->q_empty[qb]);             // no tile for this stream
+                    } else {
+                        if (ok) ok = issue_qk(x);
+                        for (int j = x; j < nt && ok; j += 2) {
+                            if (j + 2 < nt) { ok = issue_qk(j + 2); if (!ok) break; }
+                            const uint32_t vt = tiles + j;
+                            const int vs = vt % C::NV;
+                            ok = mbar_wait(&misc->p_full[x], pc & 1, misc);
+                            if (!ok) break;
+                            ok = mbar_wait(&misc->v_full[vs], (vt / C::NV) & 1, misc);
+                            if (!ok) break;
+                            if (j < 2 && unit_idx > 0) {          // the previous unit's epilogue has read O
+                                ok = mbar_wait(&misc->o_free, (unit_idx - 1) & 1, misc);
+                                if (!ok) break;
+                            }
+                            tc_fence_after();
+                            const uint32_t idesc = make_idesc(D, 1);
+                            const uint32_t v_addr = smem_u32(smem + C::OFF_V + vs * C::KV_BYTES);
+                            const int nk = (tile_cols(u, stot, j) + 15) >> 4;
+                            for (int k = 0; k < nk; ++k)
+                                tc_mma(tmem_o, desc_kmajor(p_addr + k * 32), desc_mnmajor(v_addr + k * 2048), idesc, (j >= 2 || k > 0));
+                            tc_commit(&misc->v_empty[vs]);
+                            tc_commit(&misc->p_empty[x]);
+                            if (j + 2 >= nt) tc_commit(&misc->o_full[x]);
+                            ++pc;
+                        }
+                    }
+                }
+                tiles += nt;
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                sc = __shfl_sync(0xffffffffu, sc, 0);
+                pc = __shfl_sync(0xffffffffu, pc, 0);
+            }
+            u = nxt;
+            tab = ntab;
+        }
+    } else if (warp < 4) {
+        reg_dealloc<kRegsIo>();                          // idle
+    } else {
+        // ===================================== softmax A / B ========================================
+        reg_alloc<kRegsSoftmax>();
+        const int x = warp >= 8 ? 1 : 0;                 // stream: even / odd tiles
         const int quad = warp & 3;                       // TMEM lane quadrant this warp may access
         const int row = quad * 32 + lane;                // tile row = TMEM lane
-        const int t128 = (warp - 2) * 32 + lane;         // index inside the role group (scan)
         const uint32_t lane_base = static_cast<uint32_t>(quad * 32) << 16;
-        uint32_t sc = 0, pc_full = 0, pc_wait = 0;       // S tiles consumed, P tiles produced, PV completions waited
-        uint8_t* p_tile = smem + C::OFF_P;
+        const uint32_t tmem_s = tmem + lane_base + kColS + x * kN;
+        const uint32_t tmem_o = tmem + lane_base + kColO + x * 128;
+        uint8_t* p_tile = smem + C::OFF_P + x * kPBytes;
+        float2* ml_mine = reinterpret_cast<float2*>(p_tile);                          // (max, sum) exchange area
+        const float2* ml_a = reinterpret_cast<const float2*>(smem + C::OFF_P);
+        const float2* ml_b = reinterpret_cast<const float2*>(smem + C::OFF_P + kPBytes);
+        const int b_row = row / G;                       // branch of this row inside the unit
+        uint32_t s_cnt = 0, pe_cnt = 0, unit_idx = 0;
+        uint32_t of_a = 0, of_b = 0;
         bool ok = true;
-        for (int w = blockIdx.x; w < n_units; w += gridDim.x) {
-            if (!named_bar_and(1, ok)) break;            // uniform exit of the whole role group
-            const Unit u = load_unit(p, w);
-            const int stot = suffix_scan_group(p, u, misc, 0, t128, 1);
-            const int ns = (stot + kTile - 1) / kTile;
-            const int nt = u.np + ns;
+        Unit u = load_unit(p, blockIdx.x, n_units);
+        SufTab tab = load_suftab(p, u, lane);
+        for (int w = blockIdx.x; w < n_units && ok; w += stride, ++unit_idx) {
+            const Unit nxt = load_unit(p, w + stride, n_units);
+            const SufTab ntab = load_suftab(p, nxt, lane);
+            int cs[kRounds];
+            const int stot = scan_suftab(tab, lane, cs);
+            const int nt = u.np + (stot + kN - 1) / kN;
+            // packed columns [my_cs, my_cs + my_len) hold this row's own cached tokens
+            int my_cs = 0, my_len = 0;
+#pragma unroll
+            for (int r = 0; r < kRounds; ++r) {
+                const int c = __shfl_sync(0xffffffffu, cs[r], b_row & 31);
+                const int n = __shfl_sync(0xffffffffu, tab.len[r], b_row & 31);
+                if (r == (b_row >> 5)) { my_cs = c; my_len = n; }
+            }
             const int nrows = u.nb * G;
             const bool row_valid = row < nrows;
             const bool warp_active = quad * 32 < nrows;
-            const int b = row / G, g = row - b * G;
-            int my_cs = 0, my_len = 0;
-            if (row_valid && u.with_suffix) { my_cs = misc->cs[0][b]; my_len = misc->cs[0][b + 1] - my_cs; }
-
-            float m = -INFINITY, l = 0.f;
-            for (int j = 0; j < nt && ok; ++j) {
-                const int sb = sc & 1;
-                ok = mbar_wait_warp(&misc->s_full[sb], (sc >> 1) & 1, misc);
+            const int n_mine = (nt + 1 - x) >> 1;
+            if (unit_idx > 0) {                          // P buffers and O are free again
+                ok = mbar_wait_warp(&misc->o_free, (unit_idx - 1) & 1, misc);
                 if (!ok) break;
+            }
+            float m = -INFINITY, l = 0.f;
+            for (int i = 0; i < n_mine && ok; ++i) {
+                const int j = x + 2 * i;
+                ok = mbar_wait_warp(&misc->s_full[x], s_cnt & 1, misc);
+                if (!ok) break;
+                ++s_cnt;
                 tc_fence_after();
-                int lo = 0, hi = 0;
-                if (row_valid) {
-                    if (j < u.np) { hi = min(kTile, u.key_count - j * kTile); }
-                    else {
-                        const int base = (j - u.np) * kTile;
-                        lo = max(0, my_cs - base);
-                        hi = min(kTile, my_cs + my_len - base);
-                        if (hi < lo) hi = lo;
-                    }
-                }
-                uint32_t sv[kTile];
+                uint32_t sv[kN];
                 if (warp_active) {
-                    const uint32_t ta = tmem + lane_base + sb * kTile;
-                    tmem_ld32(ta, sv); tmem_ld32(ta + 32, sv + 32); tmem_ld32(ta + 64, sv + 64); tmem_ld32(ta + 96, sv + 96);
+                    tmem_ld32(tmem_s, sv); tmem_ld32(tmem_s + 32, sv + 32);
                     tmem_ld_wait();
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&misc->s_empty[sb]);
-                ++sc;
+                if (lane == 0) mbar_arrive(&misc->s_empty[x]);
 
-                float lsum[4] = {0.f, 0.f, 0.f, 0.f};
                 bool waited = false;
                 if (warp_active) {
-                    float tmax = -INFINITY;
-                    const bool full = __all_sync(0xffffffffu, lo == 0 && hi == kTile);
-                    if (full) {
-#pragma unroll
-                        for (int c = 0; c < kTile; ++c) tmax = fmaxf(tmax, __uint_as_float(sv[c]));
+                    int lo = 0, hi;
+                    if (j < u.np) {
+                        hi = min(kN, u.key_count - j * kN);
                     } else {
+                        const int base = (j - u.np) * kN;
+                        lo = max(0, my_cs - base);
+                        hi = min(kN, my_cs + my_len - base);
+                        if (hi < lo) hi = lo;
+                    }
+                    if (!__all_sync(0xffffffffu, lo == 0 && hi == kN)) {
                         const unsigned span = static_cast<unsigned>(hi - lo);
 #pragma unroll
-                        for (int c = 0; c < kTile; ++c) {
-                            const bool v = static_cast<unsigned>(c - lo) < span;
-                            const float x = v ? __uint_as_float(sv[c]) : -INFINITY;
-                            sv[c] = __float_as_uint(x);
-                            tmax = fmaxf(tmax, x);
-                        }
+                        for (int c = 0; c < kN; ++c)
+                            if (static_cast<unsigned>(c - lo) >= span) sv[c] = 0xff800000u;   // -inf
                     }
+                    float t8[8];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) t8[c] = __uint_as_float(sv[c]);
+#pragma unroll
+                    for (int c = 8; c < kN; ++c) t8[c & 7] = fmaxf(t8[c & 7], __uint_as_float(sv[c]));
+                    float tmax = fmaxf(fmaxf(fmaxf(t8[0], t8[1]), fmaxf(t8[2], t8[3])), fmaxf(fmaxf(t8[4], t8[5]), fmaxf(t8[6], t8[7])));
                     tmax *= p.scale_log2;
-                    if (j == 0) {
+                    if (i == 0) {
                         m = tmax;
                     } else {
                         const bool grow = tmax > m + kRescaleSlack;
                         if (__any_sync(0xffffffffu, grow)) {
-                            // O must be rescaled: wait until the previous P V product has landed in TMEM
-                            ok = mbar_wait_warp(&misc->p_empty, pc_wait & 1, misc);
-                            ++pc_wait; waited = true;
+                            // O must be rescaled: wait until this stream's previous P V product has landed in TMEM
+                            ok = mbar_wait_warp(&misc->p_empty[x], pe_cnt & 1, misc);
+                            ++pe_cnt; waited = true;
                             if (ok) {
                                 tc_fence_after();
                                 const float m_new = grow ? tmax : m;
@@ -470,11 +560,11 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 #pragma unroll
                                 for (int c0 = 0; c0 < D; c0 += 32) {
                                     uint32_t ov[32];
-                                    tmem_ld32(tmem_o + lane_base + c0, ov);
+                                    tmem_ld32(tmem_o + c0, ov);
                                     tmem_ld_wait();
 #pragma unroll
                                     for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * f);
-                                    tmem_st32(tmem_o + lane_base + c0, ov);
+                                    tmem_st32(tmem_o + c0, ov);
                                 }
                                 tmem_st_wait();
                                 l *= f;
@@ -483,154 +573,123 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         }
                     }
                 }
-                if (j > 0 && !waited) {
-                    ok = ok && mbar_wait_warp(&misc->p_empty, pc_wait & 1, misc);   // previous P V has consumed the P tile
-                    ++pc_wait;
+                if (i > 0 && !waited) {
+                    ok = ok && mbar_wait_warp(&misc->p_empty[x], pe_cnt & 1, misc);   // previous P V has consumed the P tile
+                    ++pe_cnt;
                 }
+                ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 if (warp_active) {
                     const float neg_m = (m == -INFINITY) ? 0.f : -m;
                     uint8_t* prow = p_tile + row * 128;
+                    float lsum[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                    for (int kc8 = 0; kc8 < 16; ++kc8) {
+                    for (int kc8 = 0; kc8 < kN / 8; ++kc8) {
                         float e[8];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            e[i] = ex2(fmaf(__uint_as_float(sv[kc8 * 8 + i]), p.scale_log2, neg_m));
-                            lsum[i & 3] += e[i];
+                        for (int q = 0; q < 8; ++q) {
+                            e[q] = ex2(fmaf(__uint_as_float(sv[kc8 * 8 + q]), p.scale_log2, neg_m));
+                            lsum[q & 3] += e[q];
                         }
                         uint4 pk;
                         pk.x = pack_bf16(e[0], e[1]); pk.y = pack_bf16(e[2], e[3]);
                         pk.z = pack_bf16(e[4], e[5]); pk.w = pack_bf16(e[6], e[7]);
-                        *reinterpret_cast<uint4*>(prow + (kc8 >> 3) * kHalfBytes + (((kc8 & 7) ^ (row & 7)) << 4)) = pk;
+                        *reinterpret_cast<uint4*>(prow + ((kc8 ^ (row & 7)) << 4)) = pk;
                     }
                     l += (lsum[0] + lsum[1]) + (lsum[2] + lsum[3]);
                     fence_async_smem();
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&misc->p_full);
-                ++pc_full;
+                if (lane == 0) mbar_arrive(&misc->p_full[x]);
             }
-            if (!ok) continue;
+            if (!ok) break;
 
-            // -------- epilogue --------
-            if (nt > 0) {
-                ok = mbar_wait_warp(&misc->p_empty, pc_wait & 1, misc);
-                ++pc_wait;
-                if (!ok) continue;
-                tc_fence_after();
-            }
-            const int grow_row = u.row0 + b;
-            const bool store = row_valid && grow_row < p.a.max_rows;
-            if (warp_active) {
-                const int hq = u.head * G + g;
-                if (u.part_base < 0) {
-                    const float inv = l > 0.f ? 1.f / l : 0.f;
-                    __nv_bfloat16* op = p.a.o + (static_cast<int64_t>(grow_row) * p.a.g.Hq + hq) * D;
-#pragma unroll
-                    for (int c0 = 0; c0 < D; c0 += 32) {
-                        uint32_t ov[32];
-                        if (nt > 0) { tmem_ld32(tmem_o + lane_base + c0, ov); tmem_ld_wait(); }
-                        else {
-#pragma unroll
-                            for (int c = 0; c < 32; ++c) ov[c] = 0u;
-                        }
-                        if (store) {
-#pragma unroll
-                            for (int c = 0; c < 32; c += 8) {
-                                uint4 pk;
-                                pk.x = pack_bf16(__uint_as_float(ov[c + 0]) * inv, __uint_as_float(ov[c + 1]) * inv);
-                                pk.y = pack_bf16(__uint_as_float(ov[c + 2]) * inv, __uint_as_float(ov[c + 3]) * inv);
-                                pk.z = pack_bf16(__uint_as_float(ov[c + 4]) * inv, __uint_as_float(ov[c + 5]) * inv);
-                                pk.w = pack_bf16(__uint_as_float(ov[c + 6]) * inv, __uint_as_float(ov[c + 7]) * inv);
-                                *reinterpret_cast<uint4*>(op + c0 + c) = pk;
-                            }
-                        }
-                    }
-                    if (store && p.a.lse)
-                        p.a.lse[static_cast<int64_t>(grow_row) * p.a.g.Hq + hq] = l > 0.f ? (m + log2f(l)) * kLn2 : -INFINITY;
-                } else {
-                    const int64_t pr = (static_cast<int64_t>(u.part_base) + u.row_begin + b) * p.a.g.Hq + hq;
-                    float* po = p.part_o + pr * D;
-#pragma unroll
-                    for (int c0 = 0; c0 < D; c0 += 32) {
-                        uint32_t ov[32];
-                        if (nt > 0) { tmem_ld32(tmem_o + lane_base + c0, ov); tmem_ld_wait(); }
-                        else {
-#pragma unroll
-                            for (int c = 0; c < 32; ++c) ov[c] = 0u;
-                        }
-                        if (row_valid) {
-#pragma unroll
-                            for (int c = 0; c < 32; c += 4)
-                                *reinterpret_cast<uint4*>(po + c0 + c) = make_uint4(ov[c], ov[c + 1], ov[c + 2], ov[c + 3]);
-                        }
-                    }
-                    if (row_valid) { p.part_ml[pr * 2] = m; p.part_ml[pr * 2 + 1] = l; }
-                }
-            }
-            tc_fence_before();
-        }
-    } else {
-        // ========================================== gather ==========================================
-        const int t128 = (warp - 6) * 32 + lane;
-        constexpr int CHUNKS = D / 8;                    // 16-byte chunks per row and head
-        constexpr int COLS_PER_PASS = 128 / CHUNKS;
-        const int chunk = t128 % CHUNKS, col_lane = t128 / CHUNKS;
-        const int64_t cache_rows = static_cast<int64_t>(p.a.n_slots) * p.a.g.suffix_cap;
-        const int64_t tok_stride = static_cast<int64_t>(p.a.g.Hkv) * D;
-        uint32_t kc = 0, vc = 0;
-        bool ok = true;
-        for (int w = blockIdx.x; w < n_units; w += gridDim.x) {
-            if (!named_bar_and(2, ok)) break;            // uniform exit of the whole role group
-            const Unit u = load_unit(p, w);
-            const int stot = suffix_scan_group(p, u, misc, 1, t128, 2);
-            const int ns = (stot + kTile - 1) / kTile;
-            const int* cs = misc->cs[1];
-            // every ring slot is waited for in order (see the TMA producer); only suffix tiles are filled here
-            for (int j = 0; j < u.np + ns; ++j) {
-                const int ks = kc % C::NK, vs = vc % C::NV;
-                bool w_ok = mbar_wait(&misc->k_empty[ks], ((kc / C::NK) & 1) ^ 1, misc);
-                w_ok = mbar_wait(&misc->v_empty[vs], ((vc / C::NV) & 1) ^ 1, misc) && w_ok;
-                ++kc; ++vc;
-                if (j < u.np) { ok = ok && w_ok; continue; }
-                ok = named_bar_and(2, ok && w_ok);
+            // ------------------------------------ epilogue ------------------------------------
+            // both groups merge the two streams; group x writes output columns [x*D/2, (x+1)*D/2)
+            if (n_mine > 0) {                            // this stream's last P V has landed (and P is free)
+                ok = mbar_wait_warp(&misc->p_empty[x], pe_cnt & 1, misc);
+                ++pe_cnt;
                 if (!ok) break;
-                const int s = j - u.np;
-                const uint32_t k_dst = smem_u32(smem + C::OFF_K + ks * C::TILE_BYTES);
-                uint8_t* v_gen = smem + C::OFF_V + vs * C::TILE_BYTES;
-                const uint32_t v_dst = smem_u32(v_gen);
-                const int valid = min(kTile, stot - s * kTile);
-                const int padded = (valid + 15) & ~15;
-                for (int cl = col_lane; cl < padded; cl += COLS_PER_PASS) {
-                    const uint32_t off = (chunk >> 3) * kHalfBytes + cl * 128 + (((chunk & 7) ^ (cl & 7)) << 4);
-                    if (cl < valid) {
-                        const int c = s * kTile + cl;
-                        int lo_b = 0, hi_b = u.nb;               // largest b with cs[b] <= c
-                        while (hi_b - lo_b > 1) {
-                            const int mid = (lo_b + hi_b) >> 1;
-                            if (cs[mid] <= c) lo_b = mid; else hi_b = mid;
-                        }
-                        const int64_t srow = static_cast<int64_t>(p.a.suffix_off[u.row0 + lo_b]) + (c - cs[lo_b]);
-                        if (srow >= 0 && srow < cache_rows) {
-                            const int64_t e = srow * tok_stride + static_cast<int64_t>(u.head) * D + chunk * 8;
-                            cp_async16(k_dst + off, p.a.suffix_k + e);
-                            cp_async16(v_dst + off, p.a.suffix_v + e);
-                        } else {
-                            *reinterpret_cast<uint4*>(v_gen + off) = make_uint4(0, 0, 0, 0);
-                            if (p.a.dev_status) atomicOr(p.a.dev_status, HPD_S_BAD_TABLE);
+            }
+            ml_mine[row] = make_float2(m, l);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&misc->ml_full);
+            ok = mbar_wait_warp(&misc->ml_full, unit_idx & 1, misc);
+            if (!ok) break;
+            const int n_a = (nt + 1) >> 1, n_b = nt >> 1;
+            if (n_a > 0) { ok = mbar_wait_warp(&misc->o_full[0], of_a & 1, misc); ++of_a; if (!ok) break; }
+            if (n_b > 0) { ok = mbar_wait_warp(&misc->o_full[1], of_b & 1, misc); ++of_b; if (!ok) break; }
+            tc_fence_after();
+
+            const float2 sa = ml_a[row], sb = ml_b[row];
+            const float mt = fmaxf(sa.x, sb.x);
+            const float fa = sa.x == -INFINITY ? 0.f : ex2(sa.x - mt);
+            const float fb = sb.x == -INFINITY ? 0.f : ex2(sb.x - mt);
+            const float lt = fa * sa.y + fb * sb.y;
+
+            constexpr int HC = D / 2;                    // columns of this group's half
+            const int g_row = row - b_row * G;
+            const int grow_row = u.row0 + b_row;
+            const int hq = u.head * G + g_row;
+            const bool store = row_valid && grow_row < p.a.max_rows;
+            const bool final_out = u.part_base < 0;
+            const float inv = final_out ? (lt > 0.f ? 1.f / lt : 0.f) : 1.f;
+            const float ca = fa * inv, cb = fb * inv;
+            __nv_bfloat16* op = p.a.o + (static_cast<int64_t>(grow_row) * p.a.g.Hq + hq) * D + x * HC;
+            const int64_t pr = (static_cast<int64_t>(final_out ? 0 : u.part_base) + u.row_begin + b_row) * p.a.g.Hq + hq;
+            float* po = p.part_o + pr * D + x * HC;
+#pragma unroll
+            for (int c0 = 0; c0 < HC; c0 += 32) {
+                float acc[32];
+#pragma unroll
+                for (int c = 0; c < 32; ++c) acc[c] = 0.f;
+                if (warp_active) {
+                    uint32_t oa[32], ob[32];
+                    if (n_a > 0) tmem_ld32(tmem + lane_base + kColO + x * HC + c0, oa);
+                    if (n_b > 0) tmem_ld32(tmem + lane_base + kColO + 128 + x * HC + c0, ob);
+                    tmem_ld_wait();
+                    if (n_a > 0) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) acc[c] = ca * __uint_as_float(oa[c]);
+                    }
+                    if (n_b > 0) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) acc[c] = fmaf(cb, __uint_as_float(ob[c]), acc[c]);
+                    }
+                }
+                if (c0 + 32 >= HC) {                     // all TMEM reads of this unit are done
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&misc->o_free);
+                }
+                if (store) {
+                    if (final_out) {
+#pragma unroll
+                        for (int c = 0; c < 32; c += 8) {
+                            uint4 pk;
+                            pk.x = pack_bf16(acc[c + 0], acc[c + 1]);
+                            pk.y = pack_bf16(acc[c + 2], acc[c + 3]);
+                            pk.z = pack_bf16(acc[c + 4], acc[c + 5]);
+                            pk.w = pack_bf16(acc[c + 6], acc[c + 7]);
+                            *reinterpret_cast<uint4*>(op + c0 + c) = pk;
                         }
                     } else {
-                        *reinterpret_cast<uint4*>(v_gen + off) = make_uint4(0, 0, 0, 0);   // padding keys: 0 * V must stay 0
+#pragma unroll
+                        for (int c = 0; c < 32; c += 4)
+                            *reinterpret_cast<float4*>(po + c0 + c) = make_float4(acc[c], acc[c + 1], acc[c + 2], acc[c + 3]);
                     }
                 }
-                asm volatile("cp.async.commit_group;" ::: "memory");
-                asm volatile("cp.async.wait_group 0;" ::: "memory");
-                fence_async_smem();
-                named_bar(2);
-                if (t128 == 0) { mbar_arrive(&misc->k_full[ks]); mbar_arrive(&misc->v_full[vs]); }
             }
+            if (store && x == 0) {
+                if (final_out) {
+                    if (p.a.lse) p.a.lse[static_cast<int64_t>(grow_row) * p.a.g.Hq + hq] = lt > 0.f ? (mt + log2f(lt)) * kLn2 : -INFINITY;
+                } else {
+                    p.part_ml[pr * 2] = mt; p.part_ml[pr * 2 + 1] = lt;
+                }
+            }
+            u = nxt;
+            tab = ntab;
         }
     }
 
@@ -715,14 +774,14 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn()
     return fn;
 }
 
-// K/V [tokens, Hkv, D] bf16: boxes of 128 tokens x 1 head x 64 elements, 128-byte swizzle
-bool make_kv_map(CUtensorMap* m, const void* base, int D, int Hkv, long long tokens)
+// K/V [tokens, Hkv, D] bf16: boxes of box_rows tokens x 1 head x 64 elements, 128-byte swizzle
+bool make_kv_map(CUtensorMap* m, const void* base, int D, int Hkv, long long tokens, int box_rows)
 {
     auto fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[3] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(Hkv), static_cast<cuuint64_t>(tokens > 0 ? tokens : 1)};
     cuuint64_t strides[2] = {static_cast<cuuint64_t>(D) * 2, static_cast<cuuint64_t>(Hkv) * D * 2};
-    cuuint32_t box[3] = {64, 1, kTile};
+    cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(box_rows)};
     cuuint32_t es[3] = {1, 1, 1};
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -738,7 +797,7 @@ bool make_q_map(CUtensorMap* m, const void* base, int D, int G, int Hkv, long lo
                           static_cast<cuuint64_t>(rows > 0 ? rows : 1)};
     cuuint64_t strides[3] = {static_cast<cuuint64_t>(D) * 2, static_cast<cuuint64_t>(G) * D * 2,
                              static_cast<cuuint64_t>(Hkv) * G * D * 2};
-    cuuint32_t box[4] = {64, static_cast<cuuint32_t>(G), 1, static_cast<cuuint32_t>(kTile / G)};
+    cuuint32_t box[4] = {64, static_cast<cuuint32_t>(G), 1, static_cast<cuuint32_t>(kM / G)};
     cuuint32_t es[4] = {1, 1, 1, 1};
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -756,10 +815,16 @@ int launch_d(const AttnArgs& a)
     }
     const int G = a.g.Hq / a.g.Hkv;
     CUtensorMap mq, mk, mv;
+    SufMaps sm;
     const void* kbase = a.total_prefix > 0 ? static_cast<const void*>(a.prefix_k) : static_cast<const void*>(a.suffix_k);
     const void* vbase = a.total_prefix > 0 ? static_cast<const void*>(a.prefix_v) : static_cast<const void*>(a.suffix_v);
-    if (!make_q_map(&mq, a.q, D, G, a.g.Hkv, a.max_rows) || !make_kv_map(&mk, kbase, D, a.g.Hkv, a.total_prefix) ||
-        !make_kv_map(&mv, vbase, D, a.g.Hkv, a.total_prefix)) {
+    const long long cache_rows = static_cast<long long>(a.n_slots) * a.g.suffix_cap;
+    bool maps_ok = make_q_map(&mq, a.q, D, G, a.g.Hkv, a.max_rows) && make_kv_map(&mk, kbase, D, a.g.Hkv, a.total_prefix, kN) &&
+                   make_kv_map(&mv, vbase, D, a.g.Hkv, a.total_prefix, kN);
+    for (int i = 0; i < kBoxKinds && maps_ok; ++i)
+        maps_ok = make_kv_map(&sm.k[i], a.suffix_k, D, a.g.Hkv, cache_rows, 1 << i) &&
+                  make_kv_map(&sm.v[i], a.suffix_v, D, a.g.Hkv, cache_rows, 1 << i);
+    if (!maps_ok) {
         set_last_cuda_error(cudaErrorInvalidValue);
         return HPD_E_CUDA;
     }
@@ -773,7 +838,7 @@ int launch_d(const AttnArgs& a)
     p.scale_log2 = a.g.sm_scale * kLog2e;
     p.G = G;
     const int n_sm = sm_count();
-    hpd_attn_tc_kernel<D><<<n_sm, kThreads, C::SMEM, a.stream>>>(mq, mk, mv, p);
+    hpd_attn_tc_kernel<D><<<n_sm, kThreads, C::SMEM, a.stream>>>(mq, mk, mv, sm, p);
     hpd_merge_kernel<D><<<n_sm * 2, 256, 0, a.stream>>>(p, reinterpret_cast<const DocSplit*>(ws + a.lay.off_split));
     HPD_CUDA_TRY(cudaGetLastError());
     return HPD_OK;
