@@ -202,12 +202,17 @@ struct Unit {
     int np;          // prefix tiles
 };
 
-__device__ __forceinline__ Unit load_unit(const TcParams& p, int w, int n_units) {
+// Unit descriptors are fetched in two stages so that no role ever waits for a dependent load: the work
+// item of unit i+2 and, from the work item fetched one iteration earlier, the document tables of unit i+1.
+__device__ __forceinline__ WorkItem load_item(const TcParams& p, int w, int n_units) {
+    WorkItem it{};
+    if (w < n_units) it = p.work[w / p.a.g.Hkv];
+    return it;
+}
+__device__ __forceinline__ Unit make_unit(const TcParams& p, const WorkItem& it, int w, int n_units) {
     Unit u{};
     if (w >= n_units) return u;
-    const int Hkv = p.a.g.Hkv;
-    const WorkItem it = p.work[w / Hkv];
-    u.head = w % Hkv; u.key_count = it.key_count; u.part_base = it.part_base;
+    u.head = w % p.a.g.Hkv; u.key_count = it.key_count; u.part_base = it.part_base;
     u.row_begin = it.row_begin; u.nb = it.row_count; u.with_suffix = it.with_suffix;
     u.row0 = p.a.doc_active_start[it.doc] + it.row_begin;
     u.kv_row0 = p.a.doc_kv_start[it.doc] + it.key_begin;
@@ -313,11 +318,14 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         reg_dealloc<kRegsIo>();
         uint32_t qc = 0, kc = 0, vc = 0;
         bool ok = true;
-        Unit u = load_unit(p, blockIdx.x, n_units);
+        Unit u = make_unit(p, load_item(p, blockIdx.x, n_units), blockIdx.x, n_units);
         SufTab tab = load_suftab(p, u, lane);
+        Unit nxt = make_unit(p, load_item(p, blockIdx.x + stride, n_units), blockIdx.x + stride, n_units);
+        WorkItem it2 = load_item(p, blockIdx.x + 2 * stride, n_units);
         for (int w = blockIdx.x; w < n_units && ok; w += stride) {
-            const Unit nxt = load_unit(p, w + stride, n_units);
-            const SufTab ntab = load_suftab(p, nxt, lane);
+            const SufTab ntab = load_suftab(p, nxt, lane);                   // nxt was fetched one unit ago
+            const Unit nxt2 = make_unit(p, it2, w + 2 * stride, n_units);     // it2 was fetched one unit ago
+            it2 = load_item(p, w + 3 * stride, n_units);
             int cs[kRounds];
             const int stot = scan_suftab(tab, lane, cs);
             if (__any_sync(0xffffffffu, tab.bad) && lane == 0 && p.a.dev_status) atomicOr(p.a.dev_status, HPD_S_BAD_TABLE);
@@ -379,6 +387,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 }
             }
             u = nxt;
+            nxt = nxt2;
             tab = ntab;
         }
     } else if (warp < 3) {
@@ -390,11 +399,14 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         bool ok = true;
         const uint32_t p_addr = smem_u32(smem + C::OFF_P + x * kPBytes);
         const uint32_t tmem_s = tmem + kColS + x * kN, tmem_o = tmem + kColO + x * 128;
-        Unit u = load_unit(p, blockIdx.x, n_units);
+        Unit u = make_unit(p, load_item(p, blockIdx.x, n_units), blockIdx.x, n_units);
         SufTab tab = load_suftab(p, u, lane);
+        Unit nxt = make_unit(p, load_item(p, blockIdx.x + stride, n_units), blockIdx.x + stride, n_units);
+        WorkItem it2 = load_item(p, blockIdx.x + 2 * stride, n_units);
         for (int w = blockIdx.x; w < n_units && ok; w += stride, ++unit_idx) {
-            const Unit nxt = load_unit(p, w + stride, n_units);
-            const SufTab ntab = load_suftab(p, nxt, lane);
+            const SufTab ntab = load_suftab(p, nxt, lane);                   // nxt was fetched one unit ago
+            const Unit nxt2 = make_unit(p, it2, w + 2 * stride, n_units);     // it2 was fetched one unit ago
+            it2 = load_item(p, w + 3 * stride, n_units);
             int cs[kRounds];
             const int stot = scan_suftab(tab, lane, cs);
             const int nt = u.np + (stot + kN - 1) / kN;
@@ -460,6 +472,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 pc = __shfl_sync(0xffffffffu, pc, 0);
             }
             u = nxt;
+            nxt = nxt2;
             tab = ntab;
         }
     } else if (warp < 4) {
@@ -481,11 +494,14 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         uint32_t s_cnt = 0, pe_cnt = 0, unit_idx = 0;
         uint32_t of_a = 0, of_b = 0;
         bool ok = true;
-        Unit u = load_unit(p, blockIdx.x, n_units);
+        Unit u = make_unit(p, load_item(p, blockIdx.x, n_units), blockIdx.x, n_units);
         SufTab tab = load_suftab(p, u, lane);
+        Unit nxt = make_unit(p, load_item(p, blockIdx.x + stride, n_units), blockIdx.x + stride, n_units);
+        WorkItem it2 = load_item(p, blockIdx.x + 2 * stride, n_units);
         for (int w = blockIdx.x; w < n_units && ok; w += stride, ++unit_idx) {
-            const Unit nxt = load_unit(p, w + stride, n_units);
-            const SufTab ntab = load_suftab(p, nxt, lane);
+            const SufTab ntab = load_suftab(p, nxt, lane);                   // nxt was fetched one unit ago
+            const Unit nxt2 = make_unit(p, it2, w + 2 * stride, n_units);     // it2 was fetched one unit ago
+            it2 = load_item(p, w + 3 * stride, n_units);
             int cs[kRounds];
             const int stot = scan_suftab(tab, lane, cs);
             const int nt = u.np + (stot + kN - 1) / kN;
@@ -636,7 +652,6 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             const bool final_out = u.part_base < 0;
             const float inv = final_out ? (lt > 0.f ? 1.f / lt : 0.f) : 1.f;
             const float ca = fa * inv, cb = fb * inv;
-            __nv_bfloat16* op = p.a.o + (static_cast<int64_t>(grow_row) * p.a.g.Hq + hq) * D + x * HC;
             const int64_t pr = (static_cast<int64_t>(final_out ? 0 : u.part_base) + u.row_begin + b_row) * p.a.g.Hq + hq;
             float* po = p.part_o + pr * D + x * HC;
 #pragma unroll
@@ -663,22 +678,35 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&misc->o_free);
                 }
-                if (store) {
-                    if (final_out) {
+                if (final_out) {
+                    // transpose through shared memory (2 KB inside this warp's own rows of the stream's idle P tile,
+                    // past the (max, sum) exchange area): a row's 32 columns go out as one 64-byte piece, 8 rows per store
+                    uint8_t* stg = p_tile + quad * 4096 + 1024;
 #pragma unroll
-                        for (int c = 0; c < 32; c += 8) {
-                            uint4 pk;
-                            pk.x = pack_bf16(acc[c + 0], acc[c + 1]);
-                            pk.y = pack_bf16(acc[c + 2], acc[c + 3]);
-                            pk.z = pack_bf16(acc[c + 4], acc[c + 5]);
-                            pk.w = pack_bf16(acc[c + 6], acc[c + 7]);
-                            *reinterpret_cast<uint4*>(op + c0 + c) = pk;
-                        }
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 32; c += 4)
-                            *reinterpret_cast<float4*>(po + c0 + c) = make_float4(acc[c], acc[c + 1], acc[c + 2], acc[c + 3]);
+                    for (int c = 0; c < 32; c += 8) {
+                        uint4 pk;
+                        pk.x = pack_bf16(acc[c + 0], acc[c + 1]);
+                        pk.y = pack_bf16(acc[c + 2], acc[c + 3]);
+                        pk.z = pack_bf16(acc[c + 4], acc[c + 5]);
+                        pk.w = pack_bf16(acc[c + 6], acc[c + 7]);
+                        *reinterpret_cast<uint4*>(stg + lane * 64 + ((((c >> 3) ^ (lane >> 1)) & 3) << 4)) = pk;
                     }
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int rl = 8 * i + (lane >> 2), ch = lane & 3;       // row inside the warp's 32, 16-byte piece
+                        const uint4 pk = *reinterpret_cast<const uint4*>(stg + rl * 64 + (((ch ^ (rl >> 1)) & 3) << 4));
+                        const int trow = quad * 32 + rl;
+                        const int tb = trow / G, tg = trow - tb * G;
+                        const int grow = u.row0 + tb;
+                        if (trow < nrows && grow < p.a.max_rows)
+                            *reinterpret_cast<uint4*>(p.a.o + (static_cast<int64_t>(grow) * p.a.g.Hq + u.head * G + tg) * D + x * HC + c0 + ch * 8) = pk;
+                    }
+                    __syncwarp();
+                } else if (store) {
+#pragma unroll
+                    for (int c = 0; c < 32; c += 4)
+                        *reinterpret_cast<float4*>(po + c0 + c) = make_float4(acc[c], acc[c + 1], acc[c + 2], acc[c + 3]);
                 }
             }
             if (store && x == 0) {
@@ -689,6 +717,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 }
             }
             u = nxt;
+            nxt = nxt2;
             tab = ntab;
         }
     }
