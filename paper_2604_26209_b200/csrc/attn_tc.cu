@@ -47,6 +47,7 @@ constexpr uint32_t kColS = 0, kColO = 128;
 constexpr int kRegsIo = 80, kRegsSoftmax = 208;
 constexpr int kBoxKinds = 5;               // suffix boxes of 1, 2, 4, 8, 16 cache rows
 constexpr int kRounds = 4;                 // a unit has at most 128 branches: 4 rounds of 32 lanes
+constexpr int kConsumerWarps = 11;         // warps that read unit descriptors (all but the scheduler)
 
 template <int D> struct Cfg {
     static constexpr int HALVES = D / 64;
@@ -59,19 +60,9 @@ template <int D> struct Cfg {
     static constexpr int OFF_K = OFF_P + 2 * kPBytes;
     static constexpr int OFF_V = OFF_K + NK * KV_BYTES;
     static constexpr int OFF_MISC = OFF_V + NV * KV_BYTES;
-    static constexpr int SMEM = OFF_MISC + 2048 + 1024;          // + misc + slack for 1024-B alignment
+    static constexpr int SMEM = OFF_MISC + 3072;                 // + misc; the dynamic segment itself is 1024-B aligned
 };
 static_assert(Cfg<128>::SMEM <= 232448, "shared memory budget");
-
-struct Misc {
-    unsigned long long q_full[2], q_empty[2];
-    unsigned long long k_full[8], k_empty[8], v_full[8], v_empty[8];
-    unsigned long long s_full[2], s_empty[2], p_full[2], p_empty[2], o_full[2];
-    unsigned long long o_free, ml_full;
-    uint32_t tmem_base;
-    int abort_flag;
-};
-static_assert(sizeof(Misc) <= 2048, "misc block");
 
 struct SufMaps {                            // tensor maps of the branch cache, one per box height
     CUtensorMap k[kBoxKinds], v[kBoxKinds];
@@ -86,6 +77,40 @@ struct TcParams {
     float scale_log2;
     int G;
 };
+
+// ------------------------------------------------------------------------------------------------
+// Unit descriptors.  One warp (the scheduler) draws work units from the step's ticket counter, gathers
+// everything the other roles need to know about a unit -- tile counts, first rows, and per branch the
+// number of cached tokens, the first cache row and the packed column of its first token -- and publishes
+// it in one of two shared-memory slots.  Every other warp copies what it needs into registers at the start
+// of the unit and releases the slot at once, so no role ever waits for a dependent global load.
+// ------------------------------------------------------------------------------------------------
+struct UnitDesc {
+    int nt;          // tiles of the unit (prefix + suffix); -1: no more units
+    int np;          // prefix tiles
+    int stot;        // cached tokens of all branches (= packed suffix columns)
+    int head, key_count, part_base, row_begin, nb /*branches*/;
+    int row0;        // first global row
+    int kv_row0;     // first global prefix token row
+    int pad[2];
+    uint16_t cs[kM];     // per branch: packed column of its first cached token
+    uint16_t len[kM];    // per branch: cached tokens visible (0 for a bad table entry)
+    int off[kM];         // per branch: first cache row
+};
+static_assert(sizeof(UnitDesc) == 48 + 4 * kM + 4 * kM, "descriptor size");
+
+struct Misc {
+    unsigned long long q_full[2], q_empty[2];
+    unsigned long long k_full[8], k_empty[8], v_full[8], v_empty[8];
+    unsigned long long s_full[2], s_empty[2], p_full[2], p_empty[2], o_full[2];
+    unsigned long long o_free, ml_full, desc_full[2], desc_empty[2];
+    uint32_t tmem_base;
+    int abort_flag;
+    int pad[2];
+    UnitDesc desc[2];
+};
+
+static_assert(sizeof(Misc) <= 3072, "misc block");
 
 // ------------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -193,79 +218,21 @@ __device__ __forceinline__ uint32_t make_idesc(int N, int b_mn_major) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// per-unit bookkeeping shared by all roles (every role recomputes it from the same global data)
+// per-unit bookkeeping
 // ------------------------------------------------------------------------------------------------
-struct Unit {
-    int head, key_count, part_base, row_begin, nb /*branches*/, with_suffix;
-    int row0;        // first global row
-    int kv_row0;     // first global prefix token row
-    int np;          // prefix tiles
+struct Unit {        // the scalars of a descriptor, in registers
+    int nt, np, stot, head, key_count, part_base, row_begin, nb, row0, kv_row0;
 };
 
-// Unit descriptors are fetched in two stages so that no role ever waits for a dependent load: the work
-// item of unit i+2 and, from the work item fetched one iteration earlier, the document tables of unit i+1.
-__device__ __forceinline__ WorkItem load_item(const TcParams& p, int w, int n_units) {
-    WorkItem it{};
-    if (w < n_units) it = p.work[w / p.a.g.Hkv];
-    return it;
-}
-__device__ __forceinline__ Unit make_unit(const TcParams& p, const WorkItem& it, int w, int n_units) {
-    Unit u{};
-    if (w >= n_units) return u;
-    u.head = w % p.a.g.Hkv; u.key_count = it.key_count; u.part_base = it.part_base;
-    u.row_begin = it.row_begin; u.nb = it.row_count; u.with_suffix = it.with_suffix;
-    u.row0 = p.a.doc_active_start[it.doc] + it.row_begin;
-    u.kv_row0 = p.a.doc_kv_start[it.doc] + it.key_begin;
-    u.np = (it.key_count + kN - 1) / kN;
+__device__ __forceinline__ Unit read_unit(const UnitDesc& d) {
+    Unit u;
+    u.nt = d.nt; u.np = d.np; u.stot = d.stot; u.head = d.head; u.key_count = d.key_count; u.part_base = d.part_base;
+    u.row_begin = d.row_begin; u.nb = d.nb; u.row0 = d.row0; u.kv_row0 = d.kv_row0;
     return u;
 }
 
-// Branch-cache table of a unit, spread over the lanes of a warp: entry r of lane i belongs to branch
-// i + 32 r.  len = cached tokens visible to the branch (0 for a bad table entry), off = first cache row.
-struct SufTab {
-    int len[kRounds], off[kRounds];
-    int bad;
-};
-
-__device__ __forceinline__ SufTab load_suftab(const TcParams& p, const Unit& u, int lane) {
-    SufTab t;
-    t.bad = 0;
-    const int64_t cache_rows = static_cast<int64_t>(p.a.n_slots) * p.a.g.suffix_cap;
-#pragma unroll
-    for (int r = 0; r < kRounds; ++r) {
-        t.len[r] = 0; t.off[r] = 0;
-        const int b = lane + 32 * r;
-        if (u.with_suffix && b < u.nb) {
-            const int row = u.row0 + b;
-            int n = p.a.suffix_len[row] + p.a.suffix_extra;
-            n = n < 0 ? 0 : (n > p.a.g.suffix_cap ? p.a.g.suffix_cap : n);
-            const int64_t srow = p.a.suffix_off[row];
-            if (srow < 0 || srow + n > cache_rows) t.bad = 1;
-            else { t.len[r] = n; t.off[r] = static_cast<int>(srow); }
-        }
-    }
-    return t;
-}
-
-// exclusive scan of the lengths over the unit's branches (packed column of each branch's first token); returns the total
-__device__ __forceinline__ int scan_suftab(const SufTab& t, int lane, int* cs /*[kRounds]*/) {
-    int carry = 0;
-#pragma unroll
-    for (int r = 0; r < kRounds; ++r) {
-        int incl = t.len[r];
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
-        }
-        cs[r] = carry + incl - t.len[r];
-        carry += __shfl_sync(0xffffffffu, incl, 31);
-    }
-    return carry;
-}
-
-__device__ __forceinline__ int tile_cols(const Unit& u, int stot, int j) {
-    return j < u.np ? min(kN, u.key_count - j * kN) : min(kN, stot - (j - u.np) * kN);
+__device__ __forceinline__ int tile_cols(const Unit& u, int j) {
+    return j < u.np ? min(kN, u.key_count - j * kN) : min(kN, u.stot - (j - u.np) * kN);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -277,13 +244,14 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                    const __grid_constant__ CUtensorMap map_v, const __grid_constant__ SufMaps smaps, const TcParams p)
 {
     using C = Cfg<D>;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    extern __shared__ __align__(1024) uint8_t smem[];
     Misc* misc = reinterpret_cast<Misc*>(smem + C::OFF_MISC);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = p.G;
-    const int n_units = p.hdr->n_work * p.a.g.Hkv;
-    const int stride = gridDim.x;
+    if ((smem_u32(smem) & 1023u) != 0) {                 // swizzled tiles need 1024-byte alignment: refuse rather than misread
+        if (threadIdx.x == 0 && p.a.dev_status) atomicOr(p.a.dev_status, HPD_S_BAD_TABLE);
+        return;
+    }
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < 2; ++i) {
@@ -297,6 +265,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             mbar_init(&misc->v_full[i], 1); mbar_init(&misc->v_empty[i], 1);
         }
         mbar_init(&misc->o_free, 8); mbar_init(&misc->ml_full, 8);
+        for (int i = 0; i < 2; ++i) { mbar_init(&misc->desc_full[i], 1); mbar_init(&misc->desc_empty[i], kConsumerWarps); }
         misc->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -318,18 +287,19 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         reg_dealloc<kRegsIo>();
         uint32_t qc = 0, kc = 0, vc = 0;
         bool ok = true;
-        Unit u = make_unit(p, load_item(p, blockIdx.x, n_units), blockIdx.x, n_units);
-        SufTab tab = load_suftab(p, u, lane);
-        Unit nxt = make_unit(p, load_item(p, blockIdx.x + stride, n_units), blockIdx.x + stride, n_units);
-        WorkItem it2 = load_item(p, blockIdx.x + 2 * stride, n_units);
-        for (int w = blockIdx.x; w < n_units && ok; w += stride) {
-            const SufTab ntab = load_suftab(p, nxt, lane);                   // nxt was fetched one unit ago
-            const Unit nxt2 = make_unit(p, it2, w + 2 * stride, n_units);     // it2 was fetched one unit ago
-            it2 = load_item(p, w + 3 * stride, n_units);
-            int cs[kRounds];
-            const int stot = scan_suftab(tab, lane, cs);
-            if (__any_sync(0xffffffffu, tab.bad) && lane == 0 && p.a.dev_status) atomicOr(p.a.dev_status, HPD_S_BAD_TABLE);
-            const int nt = u.np + (stot + kN - 1) / kN;
+        for (uint32_t ui = 0; ok; ++ui) {
+            const int slot = ui & 1;
+            ok = mbar_wait_warp(&misc->desc_full[slot], (ui >> 1) & 1, misc);
+            if (!ok) break;
+            const UnitDesc& d = misc->desc[slot];
+            const Unit u = read_unit(d);
+            int cs[kRounds], len[kRounds], off[kRounds];
+#pragma unroll
+            for (int r = 0; r < kRounds; ++r) { cs[r] = d.cs[lane + 32 * r]; len[r] = d.len[lane + 32 * r]; off[r] = d.off[lane + 32 * r]; }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&misc->desc_empty[slot]);
+            if (u.nt < 0) break;
+            const int nt = u.nt;
             if (nt > 0) {
                 const int qb = qc & 1;
                 ok = mbar_wait_warp(&misc->q_empty[qb], ((qc >> 1) & 1) ^ 1, misc);
@@ -350,13 +320,13 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                                 tma_load_3d(tile + h * kKHalf, &pre, full, h * 64, u.head, u.kv_row0 + t * kN);
                         }
                     } else {
-                        const int c_lo = (t - u.np) * kN, c_hi = min(stot, c_lo + kN);
+                        const int c_lo = (t - u.np) * kN, c_hi = min(u.stot, c_lo + kN);
                         if (lane == 0) mbar_expect_tx(full, static_cast<uint32_t>(c_hi - c_lo) * D * 2);
 #pragma unroll
                         for (int r = 0; r < kRounds; ++r) {
-                            const int lo = max(cs[r], c_lo), hi = min(cs[r] + tab.len[r], c_hi);
+                            const int lo = max(cs[r], c_lo), hi = min(cs[r] + len[r], c_hi);
                             int n = hi - lo;
-                            int row = tab.off[r] + (lo - cs[r]);
+                            int row = off[r] + (lo - cs[r]);
                             int col = lo - c_lo;
                             while (n > 0) {
                                 const int kind = min(kBoxKinds - 1, 31 - __clz(n));
@@ -386,97 +356,185 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     __syncwarp();
                 }
             }
-            u = nxt;
-            nxt = nxt2;
-            tab = ntab;
         }
     } else if (warp < 3) {
         // ================================ MMA issuers (one per stream) ===============================
         reg_dealloc<kRegsIo>();
-        const int x = warp - 1;                          // stream: tiles x, x+2, ...
-        uint32_t qc = 0, tiles = 0, unit_idx = 0;         // units with tiles so far; tiles of earlier units
-        uint32_t sc = 0, pc = 0;                          // this stream: S tiles issued, P tiles consumed
-        bool ok = true;
-        const uint32_t p_addr = smem_u32(smem + C::OFF_P + x * kPBytes);
-        const uint32_t tmem_s = tmem + kColS + x * kN, tmem_o = tmem + kColO + x * 128;
-        Unit u = make_unit(p, load_item(p, blockIdx.x, n_units), blockIdx.x, n_units);
-        SufTab tab = load_suftab(p, u, lane);
-        Unit nxt = make_unit(p, load_item(p, blockIdx.x + stride, n_units), blockIdx.x + stride, n_units);
-        WorkItem it2 = load_item(p, blockIdx.x + 2 * stride, n_units);
-        for (int w = blockIdx.x; w < n_units && ok; w += stride, ++unit_idx) {
-            const SufTab ntab = load_suftab(p, nxt, lane);                   // nxt was fetched one unit ago
-            const Unit nxt2 = make_unit(p, it2, w + 2 * stride, n_units);     // it2 was fetched one unit ago
-            it2 = load_item(p, w + 3 * stride, n_units);
-            int cs[kRounds];
-            const int stot = scan_suftab(tab, lane, cs);
-            const int nt = u.np + (stot + kN - 1) / kN;
-            if (nt > 0) {
+        if (lane == 0) {
+            const int x = warp - 1;                      // stream: tiles x, x+2, ...
+            uint32_t qc = 0, tiles = 0;                   // units with tiles so far; tiles of earlier units
+            uint32_t sc = 0, pc = 0;                      // this stream: S tiles issued, P tiles consumed
+            bool ok = true;
+            const uint32_t p_addr = smem_u32(smem + C::OFF_P + x * kPBytes);
+            const uint32_t tmem_s = tmem + kColS + x * kN, tmem_o = tmem + kColO + x * 128;
+            for (uint32_t ui = 0; ok; ++ui) {
+                const int slot = ui & 1;
+                ok = mbar_wait(&misc->desc_full[slot], (ui >> 1) & 1, misc);
+                if (!ok) break;
+                const Unit u = read_unit(misc->desc[slot]);
+                mbar_arrive(&misc->desc_empty[slot]);
+                if (u.nt < 0) break;
+                const int nt = u.nt;
+                if (nt == 0) continue;
                 const int qb = qc & 1;
+                const uint32_t q_addr = smem_u32(smem + C::OFF_Q + qb * C::Q_BYTES);
+                ok = mbar_wait(&misc->q_full[qb], (qc >> 1) & 1, misc);
                 ++qc;
-                if (lane == 0) {
-                    const uint32_t q_addr = smem_u32(smem + C::OFF_Q + qb * C::Q_BYTES);
-                    ok = mbar_wait(&misc->q_full[qb], ((qc - 1) >> 1) & 1, misc);
-                    auto issue_qk = [&](int j) {
-                        const uint32_t kt = tiles + j;
-                        const int ks = kt % C::NK;
-                        if (!mbar_wait(&misc->k_full[ks], (kt / C::NK) & 1, misc)) return false;
-                        if (!mbar_wait(&misc->s_empty[x], (sc & 1) ^ 1, misc)) return false;
-                        tc_fence_after();
-                        const int n_pad = (tile_cols(u, stot, j) + 15) & ~15;
-                        const uint32_t idesc = make_idesc(n_pad, 0);
-                        const uint32_t k_addr = smem_u32(smem + C::OFF_K + ks * C::KV_BYTES);
+                auto issue_qk = [&](int j) {
+                    const uint32_t kt = tiles + j;
+                    const int ks = kt % C::NK;
+                    if (!mbar_wait(&misc->k_full[ks], (kt / C::NK) & 1, misc)) return false;
+                    if (!mbar_wait(&misc->s_empty[x], (sc & 1) ^ 1, misc)) return false;
+                    tc_fence_after();
+                    const int n_pad = (tile_cols(u, j) + 15) & ~15;
+                    const uint32_t idesc = make_idesc(n_pad, 0);
+                    const uint32_t k_addr = smem_u32(smem + C::OFF_K + ks * C::KV_BYTES);
 #pragma unroll
-                        for (int k = 0; k < D / 16; ++k) {
-                            const uint32_t qoff = (k >> 2) * kQHalf + (k & 3) * 32;
-                            const uint32_t koff = (k >> 2) * kKHalf + (k & 3) * 32;
-                            tc_mma(tmem_s, desc_kmajor(q_addr + qoff), desc_kmajor(k_addr + koff), idesc, k > 0);
-                        }
-                        tc_commit(&misc->k_empty[ks]);
-                        tc_commit(&misc->s_full[x]);
-                        if (j + 2 >= nt) tc_commit(&misc->q_empty[qb]);     // this stream's last use of the Q tile
-                        ++sc;
-                        return true;
-                    };
-                    if (x >= nt) {
-                        if (ok) mbar_arrive(&misc->q_empty[qb]);             // no tile for this stream
-                    } else {
-                        if (ok) ok = issue_qk(x);
-                        for (int j = x; j < nt && ok; j += 2) {
-                            if (j + 2 < nt) { ok = issue_qk(j + 2); if (!ok) break; }
-                            const uint32_t vt = tiles + j;
-                            const int vs = vt % C::NV;
-                            ok = mbar_wait(&misc->p_full[x], pc & 1, misc);
+                    for (int k = 0; k < D / 16; ++k) {
+                        const uint32_t qoff = (k >> 2) * kQHalf + (k & 3) * 32;
+                        const uint32_t koff = (k >> 2) * kKHalf + (k & 3) * 32;
+                        tc_mma(tmem_s, desc_kmajor(q_addr + qoff), desc_kmajor(k_addr + koff), idesc, k > 0);
+                    }
+                    tc_commit(&misc->k_empty[ks]);
+                    tc_commit(&misc->s_full[x]);
+                    if (j + 2 >= nt) tc_commit(&misc->q_empty[qb]);     // this stream's last use of the Q tile
+                    ++sc;
+                    return true;
+                };
+                if (x >= nt) {
+                    if (ok) mbar_arrive(&misc->q_empty[qb]);             // no tile for this stream
+                } else {
+                    if (ok) ok = issue_qk(x);
+                    for (int j = x; j < nt && ok; j += 2) {
+                        if (j + 2 < nt) { ok = issue_qk(j + 2); if (!ok) break; }
+                        const uint32_t vt = tiles + j;
+                        const int vs = vt % C::NV;
+                        ok = mbar_wait(&misc->p_full[x], pc & 1, misc);
+                        if (!ok) break;
+                        ok = mbar_wait(&misc->v_full[vs], (vt / C::NV) & 1, misc);
+                        if (!ok) break;
+                        if (j < 2 && ui > 0) {                // the previous unit's epilogue has read O
+                            ok = mbar_wait(&misc->o_free, (ui - 1) & 1, misc);
                             if (!ok) break;
-                            ok = mbar_wait(&misc->v_full[vs], (vt / C::NV) & 1, misc);
-                            if (!ok) break;
-                            if (j < 2 && unit_idx > 0) {          // the previous unit's epilogue has read O
-                                ok = mbar_wait(&misc->o_free, (unit_idx - 1) & 1, misc);
-                                if (!ok) break;
-                            }
-                            tc_fence_after();
-                            const uint32_t idesc = make_idesc(D, 1);
-                            const uint32_t v_addr = smem_u32(smem + C::OFF_V + vs * C::KV_BYTES);
-                            const int nk = (tile_cols(u, stot, j) + 15) >> 4;
-                            for (int k = 0; k < nk; ++k)
-                                tc_mma(tmem_o, desc_kmajor(p_addr + k * 32), desc_mnmajor(v_addr + k * 2048), idesc, (j >= 2 || k > 0));
-                            tc_commit(&misc->v_empty[vs]);
-                            tc_commit(&misc->p_empty[x]);
-                            if (j + 2 >= nt) tc_commit(&misc->o_full[x]);
-                            ++pc;
                         }
+                        tc_fence_after();
+                        const uint32_t idesc = make_idesc(D, 1);
+                        const uint32_t v_addr = smem_u32(smem + C::OFF_V + vs * C::KV_BYTES);
+                        const int nk = (tile_cols(u, j) + 15) >> 4;
+                        for (int k = 0; k < nk; ++k)
+                            tc_mma(tmem_o, desc_kmajor(p_addr + k * 32), desc_mnmajor(v_addr + k * 2048), idesc, (j >= 2 || k > 0));
+                        tc_commit(&misc->v_empty[vs]);
+                        tc_commit(&misc->p_empty[x]);
+                        if (j + 2 >= nt) tc_commit(&misc->o_full[x]);
+                        ++pc;
                     }
                 }
                 tiles += nt;
-                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-                sc = __shfl_sync(0xffffffffu, sc, 0);
-                pc = __shfl_sync(0xffffffffu, pc, 0);
             }
-            u = nxt;
-            nxt = nxt2;
-            tab = ntab;
         }
     } else if (warp < 4) {
-        reg_dealloc<kRegsIo>();                          // idle
+        // ========================================= scheduler ========================================
+        // Software pipeline over units, one stage per iteration, so that every global load is consumed an
+        // iteration after it was issued: ticket (i+4) -> work item (i+3) -> document tables (i+2) ->
+        // branch table (i+1) -> scan and publish (i).
+        reg_dealloc<kRegsIo>();
+        const int n_units = p.hdr->n_work * p.a.g.Hkv;
+        const int Hkv = p.a.g.Hkv;
+        const int64_t cache_rows = static_cast<int64_t>(p.a.n_slots) * p.a.g.suffix_cap;
+        uint32_t* ticket = const_cast<uint32_t*>(&p.hdr->ticket);
+        if (n_units == 0) {                              // nothing to do: publish the stop descriptor
+            if (lane == 0) { misc->desc[0].nt = -1; mbar_arrive(&misc->desc_full[0]); }
+        } else {
+        // The first five units of a CTA are fixed (unit = CTA + i * grid), which fills the pipeline without a
+        // chain of atomics; later units are drawn from the step's ticket counter, so faster SMs take more.
+        constexpr int kStatic = 5;
+        const uint32_t first_dynamic = static_cast<uint32_t>(kStatic) * gridDim.x;
+        auto draw = [&]() {                              // next unit index of this CTA (lane 0 draws, all lanes get it)
+            uint32_t t = 0;
+            if (lane == 0) t = atomicAdd(ticket, 1u);
+            t = __shfl_sync(0xffffffffu, t, 0);
+            return static_cast<int>(min(t + first_dynamic, static_cast<uint32_t>(n_units)));
+        };
+        auto fixed = [&](int i) { return static_cast<int>(min(blockIdx.x + static_cast<uint32_t>(i) * gridDim.x, static_cast<uint32_t>(n_units))); };
+        int w0 = fixed(0), w1 = fixed(1), w2 = fixed(2), w3 = fixed(3), w4 = fixed(4);
+        auto item_of = [&](int w) { return p.work[min(w, max(n_units - 1, 0)) / Hkv]; };
+        WorkItem it3 = item_of(w3), it2 = item_of(w2), it1 = item_of(w1), it0 = item_of(w0);
+        int das2 = p.a.doc_active_start[it2.doc], dks2 = p.a.doc_kv_start[it2.doc];
+        int das1 = p.a.doc_active_start[it1.doc], dks1 = p.a.doc_kv_start[it1.doc];
+        int das0 = p.a.doc_active_start[it0.doc], dks0 = p.a.doc_kv_start[it0.doc];
+        int rl1[kRounds], ro1[kRounds], rl0[kRounds], ro0[kRounds];            // raw branch tables of units i+1 and i
+        auto load_tab = [&](int w, const WorkItem& it, int das, int* rl, int* ro) {
+#pragma unroll
+            for (int r = 0; r < kRounds; ++r) {
+                const int b = lane + 32 * r;
+                rl[r] = 0; ro[r] = 0;
+                if (w < n_units && it.with_suffix && b < it.row_count) {
+                    const int row = das + it.row_begin + b;
+                    rl[r] = p.a.suffix_len[row];
+                    ro[r] = p.a.suffix_off[row];
+                }
+            }
+        };
+        load_tab(w1, it1, das1, rl1, ro1);
+        load_tab(w0, it0, das0, rl0, ro0);
+        bool ok = true;
+        for (uint32_t ui = 0; ok; ++ui) {
+            // ---- issue the next stage of every unit in flight (results are used in the next iteration) ----
+            const int w5 = draw();
+            const WorkItem it4 = item_of(w4);
+            const int das3 = p.a.doc_active_start[it3.doc], dks3 = p.a.doc_kv_start[it3.doc];
+            int rl2[kRounds], ro2[kRounds];
+            load_tab(w2, it2, das2, rl2, ro2);
+            // ---- finish unit i: clamp, validate, scan, publish ----
+            const int slot = ui & 1;
+            if (ui >= 2) {
+                ok = mbar_wait_warp(&misc->desc_empty[slot], ((ui >> 1) & 1) ^ 1, misc);
+                if (!ok) break;
+            }
+            UnitDesc& d = misc->desc[slot];
+            const bool live = w0 < n_units;
+            int carry = 0, bad = 0;
+#pragma unroll
+            for (int r = 0; r < kRounds; ++r) {
+                const int b = lane + 32 * r;
+                int n = 0, o = 0;
+                if (live && it0.with_suffix && b < it0.row_count) {
+                    n = rl0[r] + p.a.suffix_extra;
+                    n = n < 0 ? 0 : (n > p.a.g.suffix_cap ? p.a.g.suffix_cap : n);
+                    o = ro0[r];
+                    if (o < 0 || static_cast<int64_t>(o) + n > cache_rows) { bad = 1; n = 0; o = 0; }
+                }
+                int incl = n;
+#pragma unroll
+                for (int s = 1; s < 32; s <<= 1) {
+                    const int v = __shfl_up_sync(0xffffffffu, incl, s);
+                    if (lane >= s) incl += v;
+                }
+                d.cs[b] = static_cast<uint16_t>(carry + incl - n);
+                d.len[b] = static_cast<uint16_t>(n);
+                d.off[b] = o;
+                carry += __shfl_sync(0xffffffffu, incl, 31);
+            }
+            if (__any_sync(0xffffffffu, bad) && lane == 0 && p.a.dev_status) atomicOr(p.a.dev_status, HPD_S_BAD_TABLE);
+            if (lane == 0) {
+                const int np = live ? (it0.key_count + kN - 1) / kN : 0;
+                d.nt = live ? np + (carry + kN - 1) / kN : -1;
+                d.np = np; d.stot = carry;
+                d.head = w0 % Hkv; d.key_count = it0.key_count; d.part_base = it0.part_base;
+                d.row_begin = it0.row_begin; d.nb = it0.row_count;
+                d.row0 = das0 + it0.row_begin; d.kv_row0 = dks0 + it0.key_begin;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&misc->desc_full[slot]);
+            if (!live) break;
+            // ---- shift the pipeline ----
+            w0 = w1; w1 = w2; w2 = w3; w3 = w4; w4 = w5;
+            it0 = it1; it1 = it2; it2 = it3; it3 = it4;
+            das0 = das1; dks0 = dks1; das1 = das2; dks1 = dks2; das2 = das3; dks2 = dks3;
+#pragma unroll
+            for (int r = 0; r < kRounds; ++r) { rl0[r] = rl1[r]; ro0[r] = ro1[r]; rl1[r] = rl2[r]; ro1[r] = ro2[r]; }
+        }
+        }
     } else {
         // ===================================== softmax A / B ========================================
         reg_alloc<kRegsSoftmax>();
@@ -491,28 +549,20 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const float2* ml_a = reinterpret_cast<const float2*>(smem + C::OFF_P);
         const float2* ml_b = reinterpret_cast<const float2*>(smem + C::OFF_P + kPBytes);
         const int b_row = row / G;                       // branch of this row inside the unit
-        uint32_t s_cnt = 0, pe_cnt = 0, unit_idx = 0;
+        uint32_t s_cnt = 0, pe_cnt = 0;
         uint32_t of_a = 0, of_b = 0;
         bool ok = true;
-        Unit u = make_unit(p, load_item(p, blockIdx.x, n_units), blockIdx.x, n_units);
-        SufTab tab = load_suftab(p, u, lane);
-        Unit nxt = make_unit(p, load_item(p, blockIdx.x + stride, n_units), blockIdx.x + stride, n_units);
-        WorkItem it2 = load_item(p, blockIdx.x + 2 * stride, n_units);
-        for (int w = blockIdx.x; w < n_units && ok; w += stride, ++unit_idx) {
-            const SufTab ntab = load_suftab(p, nxt, lane);                   // nxt was fetched one unit ago
-            const Unit nxt2 = make_unit(p, it2, w + 2 * stride, n_units);     // it2 was fetched one unit ago
-            it2 = load_item(p, w + 3 * stride, n_units);
-            int cs[kRounds];
-            const int stot = scan_suftab(tab, lane, cs);
-            const int nt = u.np + (stot + kN - 1) / kN;
+        for (uint32_t unit_idx = 0; ok; ++unit_idx) {
+            const int slot = unit_idx & 1;
+            ok = mbar_wait_warp(&misc->desc_full[slot], (unit_idx >> 1) & 1, misc);
+            if (!ok) break;
+            const Unit u = read_unit(misc->desc[slot]);
             // packed columns [my_cs, my_cs + my_len) hold this row's own cached tokens
-            int my_cs = 0, my_len = 0;
-#pragma unroll
-            for (int r = 0; r < kRounds; ++r) {
-                const int c = __shfl_sync(0xffffffffu, cs[r], b_row & 31);
-                const int n = __shfl_sync(0xffffffffu, tab.len[r], b_row & 31);
-                if (r == (b_row >> 5)) { my_cs = c; my_len = n; }
-            }
+            const int my_cs = misc->desc[slot].cs[b_row], my_len = misc->desc[slot].len[b_row];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&misc->desc_empty[slot]);
+            if (u.nt < 0) break;
+            const int nt = u.nt;
             const int nrows = u.nb * G;
             const bool row_valid = row < nrows;
             const bool warp_active = quad * 32 < nrows;
@@ -716,9 +766,6 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     p.part_ml[pr * 2] = mt; p.part_ml[pr * 2 + 1] = lt;
                 }
             }
-            u = nxt;
-            nxt = nxt2;
-            tab = ntab;
         }
     }
 
@@ -744,6 +791,8 @@ template <int D>
 __global__ void __launch_bounds__(256)
 hpd_merge_kernel(TcParams p, const DocSplit* __restrict__ split)
 {
+    // the attention kernel drew its units from the ticket counter: rewind it for the next launch on this workspace
+    if (blockIdx.x == 0 && threadIdx.x == 0) const_cast<WsHeader*>(p.hdr)->ticket = 0;
     if (!p.hdr->any_split) return;
     const int lane = threadIdx.x & 31;
     const int Hq = p.a.g.Hq;
