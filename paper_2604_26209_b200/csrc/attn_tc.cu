@@ -4,8 +4,9 @@
 // 128/G branches of one document (rows = branches x G query heads, the M dimension) against a chunk
 // of that document's prefix, so each prefix K/V byte is read from HBM once for all of the document's
 // branches.  Keys are consumed in tiles of 64: first the prefix tiles, then tiles into which the
-// branches' own cached tokens ("suffix") are packed back to back by TMA boxes of 1..16 cache rows;
-// those tiles are masked block-diagonally (a row sees only its own branch's columns).  Even tiles
+// branches' own cached tokens ("suffix") are packed back to back, each branch padded to a multiple of
+// four columns so that one TMA box of 4..16 cache rows places it (the few rows read beyond a branch's
+// length are masked); those tiles are masked block-diagonally (a row sees only its own branch's columns).  Even tiles
 // form stream A, odd tiles stream B, each with its own MMA-issuing warp, softmax group, score
 // buffer, probability tile and output accumulator, so the two streams run as independent
 // online-softmax pipelines over one K/V stream (a split-KV inside the CTA); the epilogue merges them.
@@ -45,7 +46,8 @@ constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz
 constexpr uint32_t kColS = 0, kColO = 128;
 // registers per thread after the warpgroups have traded them (3 x 128 threads, 168 each at launch)
 constexpr int kRegsIo = 80, kRegsSoftmax = 208;
-constexpr int kBoxKinds = 5;               // suffix boxes of 1, 2, 4, 8, 16 cache rows
+constexpr int kBoxKinds = 4;               // suffix boxes of 4, 8, 12, 16 cache rows
+constexpr int kPad = 4;                    // a branch's cached tokens occupy a multiple of 4 packed columns
 constexpr int kRounds = 4;                 // a unit has at most 128 branches: 4 rounds of 32 lanes
 constexpr int kConsumerWarps = 11;         // warps that read unit descriptors (all but the scheduler)
 
@@ -324,15 +326,16 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         if (lane == 0) mbar_expect_tx(full, static_cast<uint32_t>(c_hi - c_lo) * D * 2);
 #pragma unroll
                         for (int r = 0; r < kRounds; ++r) {
-                            const int lo = max(cs[r], c_lo), hi = min(cs[r] + len[r], c_hi);
-                            int n = hi - lo;
+                            const int plen = (len[r] + kPad - 1) & ~(kPad - 1);
+                            const int lo = max(cs[r], c_lo), hi = min(cs[r] + plen, c_hi);
+                            int n = hi - lo;                         // a multiple of 4: all segment ends and tile ends are
                             int row = off[r] + (lo - cs[r]);
                             int col = lo - c_lo;
                             while (n > 0) {
-                                const int kind = min(kBoxKinds - 1, 31 - __clz(n));
+                                const int h4 = min(n, 4 * kBoxKinds);
                                 for (int h = 0; h < C::HALVES; ++h)
-                                    tma_load_3d(tile + h * kKHalf + col * 128, &suf[kind], full, h * 64, u.head, row);
-                                row += 1 << kind; col += 1 << kind; n -= 1 << kind;
+                                    tma_load_3d(tile + h * kKHalf + col * 128, &suf[h4 / 4 - 1], full, h * 64, u.head, row);
+                                row += h4; col += h4; n -= h4;
                             }
                         }
                     }
@@ -504,13 +507,14 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     o = ro0[r];
                     if (o < 0 || static_cast<int64_t>(o) + n > cache_rows) { bad = 1; n = 0; o = 0; }
                 }
-                int incl = n;
+                const int np4 = (n + kPad - 1) & ~(kPad - 1);        // columns the branch occupies
+                int incl = np4;
 #pragma unroll
                 for (int s = 1; s < 32; s <<= 1) {
                     const int v = __shfl_up_sync(0xffffffffu, incl, s);
                     if (lane >= s) incl += v;
                 }
-                d.cs[b] = static_cast<uint16_t>(carry + incl - n);
+                d.cs[b] = static_cast<uint16_t>(carry + incl - np4);
                 d.len[b] = static_cast<uint16_t>(n);
                 d.off[b] = o;
                 carry += __shfl_sync(0xffffffffu, incl, 31);
@@ -900,8 +904,8 @@ int launch_d(const AttnArgs& a)
     bool maps_ok = make_q_map(&mq, a.q, D, G, a.g.Hkv, a.max_rows) && make_kv_map(&mk, kbase, D, a.g.Hkv, a.total_prefix, kN) &&
                    make_kv_map(&mv, vbase, D, a.g.Hkv, a.total_prefix, kN);
     for (int i = 0; i < kBoxKinds && maps_ok; ++i)
-        maps_ok = make_kv_map(&sm.k[i], a.suffix_k, D, a.g.Hkv, cache_rows, 1 << i) &&
-                  make_kv_map(&sm.v[i], a.suffix_v, D, a.g.Hkv, cache_rows, 1 << i);
+        maps_ok = make_kv_map(&sm.k[i], a.suffix_k, D, a.g.Hkv, cache_rows, 4 * (i + 1)) &&
+                  make_kv_map(&sm.v[i], a.suffix_v, D, a.g.Hkv, cache_rows, 4 * (i + 1));
     if (!maps_ok) {
         set_last_cuda_error(cudaErrorInvalidValue);
         return HPD_E_CUDA;
