@@ -714,17 +714,18 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 #pragma unroll
                 for (int c = 0; c < 32; ++c) acc[c] = 0.f;
                 if (warp_active) {
-                    uint32_t oa[32], ob[32];
-                    if (n_a > 0) tmem_ld32(tmem + lane_base + kColO + x * HC + c0, oa);
-                    if (n_b > 0) tmem_ld32(tmem + lane_base + kColO + 128 + x * HC + c0, ob);
-                    tmem_ld_wait();
+                    uint32_t ov[32];
                     if (n_a > 0) {
+                        tmem_ld32(tmem + lane_base + kColO + x * HC + c0, ov);
+                        tmem_ld_wait();
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) acc[c] = ca * __uint_as_float(oa[c]);
+                        for (int c = 0; c < 32; ++c) acc[c] = ca * __uint_as_float(ov[c]);
                     }
                     if (n_b > 0) {
+                        tmem_ld32(tmem + lane_base + kColO + 128 + x * HC + c0, ov);
+                        tmem_ld_wait();
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) acc[c] = fmaf(cb, __uint_as_float(ob[c]), acc[c]);
+                        for (int c = 0; c < 32; ++c) acc[c] = fmaf(cb, __uint_as_float(ov[c]), acc[c]);
                     }
                 }
                 if (c0 + 32 >= HC) {                     // all TMEM reads of this unit are done
