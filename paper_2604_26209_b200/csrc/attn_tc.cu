@@ -234,7 +234,9 @@ __device__ __forceinline__ Unit read_unit(const UnitDesc& d) {
 }
 
 __device__ __forceinline__ int tile_cols(const Unit& u, int j) {
-    return j < u.np ? min(kN, u.key_count - j * kN) : min(kN, u.stot - (j - u.np) * kN);
+    const int ns = u.nt - u.np;                      // suffix tiles come first: their many small copies are then
+    return j < ns ? min(kN, u.stot - j * kN)         // issued while the previous unit is still in its epilogue
+                  : min(kN, u.key_count - (j - ns) * kN);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -315,14 +317,15 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 // One tile: a prefix tile is two boxes issued by lane 0; a suffix tile is packed from boxes of
                 // 1..16 cache rows, every lane placing the part of its branches that falls into the tile.
                 auto fill = [&](int t, uint8_t* tile, unsigned long long* full, const CUtensorMap& pre, const CUtensorMap* suf) {
-                    if (t < u.np) {
+                    const int ns = nt - u.np;
+                    if (t >= ns) {
                         if (lane == 0) {
                             mbar_expect_tx(full, C::KV_BYTES);
                             for (int h = 0; h < C::HALVES; ++h)
-                                tma_load_3d(tile + h * kKHalf, &pre, full, h * 64, u.head, u.kv_row0 + t * kN);
+                                tma_load_3d(tile + h * kKHalf, &pre, full, h * 64, u.head, u.kv_row0 + (t - ns) * kN);
                         }
                     } else {
-                        const int c_lo = (t - u.np) * kN, c_hi = min(u.stot, c_lo + kN);
+                        const int c_lo = t * kN, c_hi = min(u.stot, c_lo + kN);
                         if (lane == 0) mbar_expect_tx(full, static_cast<uint32_t>(c_hi - c_lo) * D * 2);
 #pragma unroll
                         for (int r = 0; r < kRounds; ++r) {
@@ -594,10 +597,11 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 bool waited = false;
                 if (warp_active) {
                     int lo = 0, hi;
-                    if (j < u.np) {
-                        hi = min(kN, u.key_count - j * kN);
+                    const int ns = nt - u.np;
+                    if (j >= ns) {
+                        hi = min(kN, u.key_count - (j - ns) * kN);
                     } else {
-                        const int base = (j - u.np) * kN;
+                        const int base = j * kN;
                         lo = max(0, my_cs - base);
                         hi = min(kN, my_cs + my_len - base);
                         if (hi < lo) hi = lo;
@@ -618,7 +622,9 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     if (i == 0) {
                         m = tmax;
                     } else {
-                        const bool grow = tmax > m + kRescaleSlack;
+                        const bool fresh = m == -INFINITY;       // nothing visible so far: O row is still exactly zero
+                        if (fresh) m = tmax;
+                        const bool grow = !fresh && tmax > m + kRescaleSlack;
                         if (__any_sync(0xffffffffu, grow)) {
                             // O must be rescaled: wait until this stream's previous P V product has landed in TMEM
                             ok = mbar_wait_warp(&misc->p_empty[x], pe_cnt & 1, misc);
