@@ -241,14 +241,9 @@ def run_ours(args):
     barrier()
     ms_e2e = e0.elapsed_time(e1)
 
-    # ---- max over ranks ------------------------------------------------------------------------------------
-    times = torch.tensor([ms_total, ms_e2e, ms_attn], dtype=torch.float64, device="cuda")
-    tokens = torch.tensor([float(n)], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-        dist.all_reduce(tokens, op=dist.ReduceOp.SUM)
-    ms_total, ms_e2e, ms_attn_max = (float(x) for x in times.tolist())
-    tok_all = float(tokens.item())
+    # ---- max over ranks (time), sum over ranks (rows) ----------------------------------------------------------
+    from paper_2604_26209_b200.dist import reduce_timing
+    (ms_total, ms_e2e, ms_attn_max), tok_all = reduce_timing([ms_total, ms_e2e, ms_attn], n, device="cuda")
 
     if rank == 0:
         peaks = measured_peaks()
@@ -266,6 +261,32 @@ def run_ours(args):
             cpu = {"value": rows_done / t_cpu, "unit": UNIT, "cores": thr, "kind": "oracle",
                    "sample": f"{rows_done} rows ({args.cpu_rows} evenly spaced rows of the {n}-row step per pass), "
                              f"{t_cpu:.1f} s of oracle time"}
+        comparison = None
+        if world == 1 and not args.no_comparison:
+            # the in-repo comparison: every branch with a private physical copy of [prefix ; branch tokens]
+            free_b, _ = torch.cuda.mem_get_info()
+            row_b = s.geom.Hkv * s.geom.D * 2 * 2
+            need = int((s.doc_prefix_len[s.slot_doc()[s.slot_alive.astype(bool)]].astype(np.int64)
+                        + s.slot_depth[s.slot_alive.astype(bool)] + 1).sum()) * row_b
+            rows_std = n if need < 0.6 * free_b else max(1, int(n * 0.6 * free_b / need))
+            dup = runtime.DupBatch(db, include_new=True, rows=rows_std)
+            for _ in range(2):
+                dup.attn(db.q)
+            c0 = torch.cuda.Event(enable_timing=True); c1 = torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            c0.record(stream)
+            for _ in range(3):
+                dup.attn(db.q)
+            c1.record(stream)
+            torch.cuda.synchronize()
+            ms_std = c0.elapsed_time(c1) / 3 * (n / dup.n)          # linear in rows: no sharing between sequences
+            std_bytes = dup.total_tokens * row_b * (n / dup.n) + ab["qo"]
+            comparison = {"kernel": "std_attn_decode (duplicated prefix)", "ms_per_launch": ms_std,
+                          "rows_timed": dup.n, "rows_total": n,
+                          "hbm_frac_of_measured": std_bytes / (ms_std * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                          "algorithmic_bytes": int(std_bytes), "bytes_ratio_std_over_hpd": std_bytes / ab["attn"],
+                          "speedup_hpd_over_std": ms_std / ms_attn}
+            del dup
         traffic = None
         tp = os.path.join(ROOT, "profiles", "traffic.json")
         if os.path.exists(tp):
@@ -277,7 +298,7 @@ def run_ours(args):
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": s.name, "prompts_per_gpu": s.n_prompts, "branches_per_prompt": 96,
                        "docs_per_prompt": s.docs_per_prompt, "n_active_per_gpu": n, "geometry": "Hq32/Hkv8/D128",
-                       "layers": 1, "l2": "inputs larger than L2 (851 MB touched per step vs 126 MB L2); no flush",
+                       "layers": 1, "l2": f"inputs larger than L2 ({ab['attn'] / 1e6:.0f} MB touched per step vs 126 MB L2); no flush",
                        "attn_impl": os.environ.get("HPD_ATTN_IMPL", "default")},
             "clocks": clocks,
             "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
@@ -289,7 +310,7 @@ def run_ours(args):
                          "frac_of_nominal_8TBs": ach / 8000.0, "tensor_tflops_algorithmic": tflops,
                          "tensor_frac_of_measured_bf16": tflops / peaks["bf16_tflops"]},
             "breakdown_ms": {"meta_rope_append": ms_pre, "attn": ms_attn},
-            "cpu_baseline": cpu, "dev_status": status,
+            "cpu_baseline": cpu, "comparison": comparison, "dev_status": status,
         }
         print(json.dumps(out))
     if world > 1:
@@ -306,6 +327,7 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=2048)
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-comparison", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
