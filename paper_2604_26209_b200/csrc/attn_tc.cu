@@ -67,7 +67,8 @@ template <int D> struct Cfg {
 static_assert(Cfg<128>::SMEM <= 232448, "shared memory budget");
 
 struct SufMaps {                            // tensor maps of the branch cache, one per box height
-    CUtensorMap k[kBoxKinds], v[kBoxKinds];
+    CUtensorMap k[kBoxKinds];               // 4, 8, 12, 16 rows
+    CUtensorMap v[16];                      // 1 .. 16 rows
 };
 
 struct TcParams {
@@ -314,9 +315,12 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         tma_load_4d(smem + C::OFF_Q + qb * C::Q_BYTES + h * kQHalf, &map_q, &misc->q_full[qb], h * 64, 0, u.head, u.row0);
                 }
                 ++qc;
-                // One tile: a prefix tile is two boxes issued by lane 0; a suffix tile is packed from boxes of
-                // 1..16 cache rows, every lane placing the part of its branches that falls into the tile.
-                auto fill = [&](int t, uint8_t* tile, unsigned long long* full, const CUtensorMap& pre, const CUtensorMap* suf) {
+                // One tile: a prefix tile is two boxes issued by lane 0; a suffix tile is packed from one box per
+                // branch (and half), every lane placing the part of its branches that falls into the tile.  K boxes
+                // are 4, 8, 12 or 16 rows high and may read up to three rows past the branch's length (their columns
+                // are masked); V boxes have the exact height, because whatever lies beyond a branch's length in the
+                // cache -- possibly NaN -- would otherwise be multiplied by a zero probability.
+                auto fill = [&](int t, uint8_t* tile, unsigned long long* full, const CUtensorMap& pre, const CUtensorMap* suf, bool exact) {
                     const int ns = nt - u.np;
                     if (t >= ns) {
                         if (lane == 0) {
@@ -326,19 +330,27 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         }
                     } else {
                         const int c_lo = t * kN, c_hi = min(u.stot, c_lo + kN);
-                        if (lane == 0) mbar_expect_tx(full, static_cast<uint32_t>(c_hi - c_lo) * D * 2);
+                        int rows_mine = 0;
 #pragma unroll
                         for (int r = 0; r < kRounds; ++r) {
-                            const int plen = (len[r] + kPad - 1) & ~(kPad - 1);
+                            const int plen = exact ? len[r] : (len[r] + kPad - 1) & ~(kPad - 1);
+                            rows_mine += max(0, min(cs[r] + plen, c_hi) - max(cs[r], c_lo));
+                        }
+                        const int rows_all = __reduce_add_sync(0xffffffffu, rows_mine);
+                        if (lane == 0) mbar_expect_tx(full, static_cast<uint32_t>(rows_all) * D * 2);
+#pragma unroll
+                        for (int r = 0; r < kRounds; ++r) {
+                            const int plen = exact ? len[r] : (len[r] + kPad - 1) & ~(kPad - 1);
                             const int lo = max(cs[r], c_lo), hi = min(cs[r] + plen, c_hi);
-                            int n = hi - lo;                         // a multiple of 4: all segment ends and tile ends are
+                            int n = hi - lo;
                             int row = off[r] + (lo - cs[r]);
                             int col = lo - c_lo;
                             while (n > 0) {
-                                const int h4 = min(n, 4 * kBoxKinds);
+                                const int hb = min(n, 16);
+                                const CUtensorMap* m = exact ? &suf[hb - 1] : &suf[hb / 4 - 1];
                                 for (int h = 0; h < C::HALVES; ++h)
-                                    tma_load_3d(tile + h * kKHalf + col * 128, &suf[h4 / 4 - 1], full, h * 64, u.head, row);
-                                row += h4; col += h4; n -= h4;
+                                    tma_load_3d(tile + h * kKHalf + col * 128, m, full, h * 64, u.head, row);
+                                row += hb; col += hb; n -= hb;
                             }
                         }
                     }
@@ -349,14 +361,14 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         const int ks = kc % C::NK;
                         ok = mbar_wait_warp(&misc->k_empty[ks], ((kc / C::NK) & 1) ^ 1, misc);
                         if (!ok) break;
-                        fill(t, smem + C::OFF_K + ks * C::KV_BYTES, &misc->k_full[ks], map_k, smaps.k);
+                        fill(t, smem + C::OFF_K + ks * C::KV_BYTES, &misc->k_full[ks], map_k, smaps.k, false);
                         ++kc;
                     }
                     if (t >= 2) {
                         const int vs = vc % C::NV;
                         ok = mbar_wait_warp(&misc->v_empty[vs], ((vc / C::NV) & 1) ^ 1, misc);
                         if (!ok) break;
-                        fill(t - 2, smem + C::OFF_V + vs * C::KV_BYTES, &misc->v_full[vs], map_v, smaps.v);
+                        fill(t - 2, smem + C::OFF_V + vs * C::KV_BYTES, &misc->v_full[vs], map_v, smaps.v, true);
                         ++vc;
                     }
                     __syncwarp();
@@ -903,20 +915,44 @@ int launch_d(const AttnArgs& a)
         attr_set = true;
     }
     const int G = a.g.Hq / a.g.Hkv;
-    CUtensorMap mq, mk, mv;
-    SufMaps sm;
+    // Tensor maps depend only on the tensors' addresses and extents: a decode loop calls with the same ones step
+    // after step and layer after layer, so each thread keeps the maps of its last few distinct argument sets.
+    struct MapKey {
+        const void *q, *pk, *pv, *sk, *sv;
+        long long max_rows, total_prefix, cache_rows;
+        int Hkv, G;
+        bool operator==(const MapKey& o) const {
+            return q == o.q && pk == o.pk && pv == o.pv && sk == o.sk && sv == o.sv && max_rows == o.max_rows &&
+                   total_prefix == o.total_prefix && cache_rows == o.cache_rows && Hkv == o.Hkv && G == o.G;
+        }
+    };
+    struct MapSet { MapKey key; CUtensorMap mq, mk, mv; SufMaps sm; bool valid = false; };
+    constexpr int kCached = 64;
+    static thread_local MapSet cache[kCached];
+    static thread_local unsigned next_victim = 0;
     const void* kbase = a.total_prefix > 0 ? static_cast<const void*>(a.prefix_k) : static_cast<const void*>(a.suffix_k);
     const void* vbase = a.total_prefix > 0 ? static_cast<const void*>(a.prefix_v) : static_cast<const void*>(a.suffix_v);
     const long long cache_rows = static_cast<long long>(a.n_slots) * a.g.suffix_cap;
-    bool maps_ok = make_q_map(&mq, a.q, D, G, a.g.Hkv, a.max_rows) && make_kv_map(&mk, kbase, D, a.g.Hkv, a.total_prefix, kN) &&
-                   make_kv_map(&mv, vbase, D, a.g.Hkv, a.total_prefix, kN);
-    for (int i = 0; i < kBoxKinds && maps_ok; ++i)
-        maps_ok = make_kv_map(&sm.k[i], a.suffix_k, D, a.g.Hkv, cache_rows, 4 * (i + 1)) &&
-                  make_kv_map(&sm.v[i], a.suffix_v, D, a.g.Hkv, cache_rows, 4 * (i + 1));
-    if (!maps_ok) {
-        set_last_cuda_error(cudaErrorInvalidValue);
-        return HPD_E_CUDA;
+    const MapKey key{a.q, kbase, vbase, a.suffix_k, a.suffix_v, a.max_rows, a.total_prefix, cache_rows, a.g.Hkv, G};
+    MapSet* ms = nullptr;
+    for (int i = 0; i < kCached && !ms; ++i)
+        if (cache[i].valid && cache[i].key == key) ms = &cache[i];
+    if (!ms) {
+        ms = &cache[next_victim++ % kCached];
+        ms->valid = false;
+        bool maps_ok = make_q_map(&ms->mq, a.q, D, G, a.g.Hkv, a.max_rows) && make_kv_map(&ms->mk, kbase, D, a.g.Hkv, a.total_prefix, kN) &&
+                       make_kv_map(&ms->mv, vbase, D, a.g.Hkv, a.total_prefix, kN);
+        for (int i = 0; i < kBoxKinds && maps_ok; ++i) maps_ok = make_kv_map(&ms->sm.k[i], a.suffix_k, D, a.g.Hkv, cache_rows, 4 * (i + 1));
+        for (int i = 0; i < 16 && maps_ok; ++i) maps_ok = make_kv_map(&ms->sm.v[i], a.suffix_v, D, a.g.Hkv, cache_rows, i + 1);
+        if (!maps_ok) {
+            set_last_cuda_error(cudaErrorInvalidValue);
+            return HPD_E_CUDA;
+        }
+        ms->key = key;
+        ms->valid = true;
     }
+    const CUtensorMap &mq = ms->mq, &mk = ms->mk, &mv = ms->mv;
+    const SufMaps& sm = ms->sm;
     TcParams p{};
     p.a = a;
     char* ws = static_cast<char*>(a.workspace);
