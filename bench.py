@@ -317,6 +317,75 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_loop(args):
+    """Decode loop: 32 layers x up to 32 steps over the main structure with ragged retirement (end-of-value lengths
+    min(Geom(1/8), 32)).  Per step: hpd_build_meta once, then per layer hpd_rope -> hpd_kv_append -> hpd_attn_decode
+    on that layer's own prefix and branch caches.  Caches are filled on the device (torch.randn, seeded): 43 GB."""
+    import torch
+    from paper_2604_26209_b200 import binding as B
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        raise SystemExit("--workload loop is a single-GPU workload")
+    torch.cuda.set_device(0)
+    B.load()
+    s = synth.config_loop(n_prompts=args.loop_prompts, seed=0)
+    g, dev, L = s.geom, "cuda", args.layers
+    gen = torch.Generator(device=dev); gen.manual_seed(0)
+    rnd = lambda *shape: torch.randn(*shape, device=dev, dtype=torch.float32, generator=gen).to(torch.bfloat16)
+    kv = g.Hkv * g.D
+    pre_k = [rnd(s.total_prefix, kv) for _ in range(L)]; pre_v = [rnd(s.total_prefix, kv) for _ in range(L)]
+    suf_k = [torch.zeros(s.n_slots * g.suffix_cap, kv, dtype=torch.bfloat16, device=dev) for _ in range(L)]
+    suf_v = [torch.zeros_like(suf_k[0]) for _ in range(L)]
+    q = [rnd(s.n_slots, g.Hq * g.D) for _ in range(2)]
+    kn = [rnd(s.n_slots, kv) for _ in range(2)]; vn = [rnd(s.n_slots, kv) for _ in range(2)]
+    o = torch.zeros(s.n_slots, g.Hq * g.D, dtype=torch.bfloat16, device=dev)
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    L_d, cnt, eos = i32(s.doc_prefix_len), i32(s.doc_branch_cnt), i32(s.eos_len)
+    depth = torch.zeros(s.n_slots, dtype=torch.int32, device=dev)
+    alive = torch.ones(s.n_slots, dtype=torch.uint8, device=dev)
+    meta = B.MetaTables.alloc(g, s.n_docs, s.n_slots, s.total_prefix, dev)
+    steps = int(s.eos_len.max())
+    n_act = [int((s.eos_len > t).sum()) for t in range(steps)]
+    stream = torch.cuda.current_stream()
+
+    def one_step(t):
+        # caller-side state of the loop (which branches are still decoding, how deep they are)
+        torch.minimum(eos, torch.full_like(eos, t), out=depth)
+        alive.copy_((eos > t).to(torch.uint8))
+        B.hpd_build_meta(g, s.n_docs, s.n_slots, L_d, cnt, depth, alive, 0, meta)
+        for l in range(L):
+            b = (t + l) & 1
+            B.hpd_rope(g, s.n_slots, meta.n_active, meta.pos_id, q[b], kn[b])
+            B.hpd_kv_append(g, s.n_slots, s.n_slots, meta.n_active, meta.suffix_off, meta.suffix_len, kn[b], vn[b],
+                            suf_k[l], suf_v[l], meta.dev_status)
+            B.hpd_attn_decode(g, s.n_docs, s.n_slots, s.n_slots, s.total_prefix, q[b], pre_k[l], pre_v[l], suf_k[l],
+                              suf_v[l], L_d, meta, True, o, None)
+
+    for t in range(min(3, steps)):
+        one_step(t)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0); sampler.start(); time.sleep(0.3)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    ev[0].record(stream)
+    for t in range(steps):
+        one_step(t)
+        ev[t + 1].record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = [ev[t].elapsed_time(ev[t + 1]) for t in range(steps)]
+    total_ms = ev[0].elapsed_time(ev[steps])
+    tokens = sum(n_act)
+    print(json.dumps({
+        "metric": METRIC, "value": tokens / (total_ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": 3,
+        "ms_per_step": total_ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic", "config": {"workload": f"{s.name}_L{L}", "layers": L, "prompts": s.n_prompts,
+                                        "branches_per_prompt": 96, "suffix_cap": g.suffix_cap,
+                                        "l2": "inputs larger than L2 (every layer has its own caches); no flush"},
+        "clocks": clocks, "gpu_launches": steps * (3 + 4 * L), "dev_status": int(meta.dev_status.item()),
+        "per_layer_branch_tokens_per_s": tokens * L / (total_ms * 1e-3),
+        "series": [{"step": t, "n_active": n_act[t], "ms": ms[t]} for t in range(steps)],
+    }))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -328,10 +397,14 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-comparison", action="store_true")
+    ap.add_argument("--layers", type=int, default=32)
+    ap.add_argument("--loop-prompts", type=int, default=64)
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    if args.impl == "reference":
+    if args.workload == "loop" and args.impl != "reference":
+        run_loop(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
