@@ -173,10 +173,13 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 __device__ __forceinline__ void tc_commit(unsigned long long* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+// One tcgen05.mma; the two shared-memory descriptors are given as their low words (address and LBO fields, see
+// below), the high word is the same for every operand of this kernel.
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+                 "mov.b64 da, {%1, %5};\n\tmov.b64 db, {%2, %5};\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(0x40004040u) : "memory");
 }
 
 #define HPD_R8(a, o) "=r"(a[o + 0]), "=r"(a[o + 1]), "=r"(a[o + 2]), "=r"(a[o + 3]), "=r"(a[o + 4]), "=r"(a[o + 5]), "=r"(a[o + 6]), "=r"(a[o + 7])
@@ -203,17 +206,15 @@ __device__ __forceinline__ float ex2(float x) {
 template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
-// Shared-memory matrix descriptors (128-byte swizzle; version field = 1).
-//   K-major  (Q, K, P): rows of 128 B; groups of 8 rows 1024 B apart (SBO); LBO unused.
-//   MN-major (V):       rows (keys) of 128 B holding 64 head-dim elements; 8-key groups 1024 B apart
-//                       (SBO); the next 64 head-dim elements one tile half further (LBO).
-__device__ __forceinline__ uint64_t desc_kmajor(uint32_t saddr) {
-    return static_cast<uint64_t>((saddr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
-}
-__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr) {
-    return static_cast<uint64_t>((saddr >> 4) & 0x3FFF) | (static_cast<uint64_t>(kKHalf >> 4) << 16) | (64ull << 32) |
-           (1ull << 46) | (2ull << 61);
-}
+// Shared-memory matrix descriptors (128-byte swizzle; version field = 1).  High word, common to all operands:
+// SBO = 1024 B (groups of 8 rows), version 1, swizzle mode 2 (128 B) = 0x40004040.  Low word: address / 16 in bits
+// 0-13 and LBO / 16 in bits 16-29.  Shared-memory addresses are below 2^18, so moving a descriptor by a multiple
+// of 16 bytes inside a tile is a plain addition to the low word.
+//   K-major  (Q, K, P): rows of 128 B; LBO unused (1).
+//   MN-major (V):       rows (keys) of 128 B holding 64 head-dim elements; the next 64 head-dim elements one tile
+//                       half further (LBO).
+__device__ __forceinline__ uint32_t desc_lo_kmajor(uint32_t saddr) { return (saddr >> 4) | (1u << 16); }
+__device__ __forceinline__ uint32_t desc_lo_mnmajor(uint32_t saddr) { return (saddr >> 4) | (static_cast<uint32_t>(kKHalf >> 4) << 16); }
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N given; B either K-major (Q K^T) or MN-major (P V).
 __device__ __forceinline__ uint32_t make_idesc(int N, int b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(b_mn_major) << 16) |
@@ -232,12 +233,6 @@ __device__ __forceinline__ Unit read_unit(const UnitDesc& d) {
     u.nt = d.nt; u.np = d.np; u.stot = d.stot; u.head = d.head; u.key_count = d.key_count; u.part_base = d.part_base;
     u.row_begin = d.row_begin; u.nb = d.nb; u.row0 = d.row0; u.kv_row0 = d.kv_row0;
     return u;
-}
-
-__device__ __forceinline__ int tile_cols(const Unit& u, int j) {
-    const int ns = u.nt - u.np;                      // suffix tiles come first: their many small copies are then
-    return j < ns ? min(kN, u.stot - j * kN)         // issued while the previous unit is still in its epilogue
-                  : min(kN, u.key_count - (j - ns) * kN);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -395,23 +390,26 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 const int nt = u.nt;
                 if (nt == 0) continue;
                 const int qb = qc & 1;
-                const uint32_t q_addr = smem_u32(smem + C::OFF_Q + qb * C::Q_BYTES);
+                const uint32_t q_lo = desc_lo_kmajor(smem_u32(smem + C::OFF_Q + qb * C::Q_BYTES));
+                const int ns = nt - u.np;
+                // columns of tile j: only the last suffix tile and the last prefix tile can be partial
+                const int last_s = u.stot - (ns - 1) * kN, last_p = u.key_count - (u.np - 1) * kN;
+                auto cols16 = [&](int j) { return ((j == ns - 1 ? last_s : (j == nt - 1 ? last_p : kN)) + 15) >> 4; };
                 ok = mbar_wait(&misc->q_full[qb], (qc >> 1) & 1, misc);
                 ++qc;
                 auto issue_qk = [&](int j) {
                     const uint32_t kt = tiles + j;
                     const int ks = kt % C::NK;
+                    const uint32_t idesc = make_idesc(cols16(j) << 4, 0);
+                    const uint32_t k_lo = desc_lo_kmajor(smem_u32(smem + C::OFF_K)) + ks * (C::KV_BYTES >> 4);
                     if (!mbar_wait(&misc->k_full[ks], (kt / C::NK) & 1, misc)) return false;
                     if (!mbar_wait(&misc->s_empty[x], (sc & 1) ^ 1, misc)) return false;
                     tc_fence_after();
-                    const int n_pad = (tile_cols(u, j) + 15) & ~15;
-                    const uint32_t idesc = make_idesc(n_pad, 0);
-                    const uint32_t k_addr = smem_u32(smem + C::OFF_K + ks * C::KV_BYTES);
 #pragma unroll
                     for (int k = 0; k < D / 16; ++k) {
-                        const uint32_t qoff = (k >> 2) * kQHalf + (k & 3) * 32;
-                        const uint32_t koff = (k >> 2) * kKHalf + (k & 3) * 32;
-                        tc_mma(tmem_s, desc_kmajor(q_addr + qoff), desc_kmajor(k_addr + koff), idesc, k > 0);
+                        const uint32_t qoff = ((k >> 2) * kQHalf + (k & 3) * 32) >> 4;
+                        const uint32_t koff = ((k >> 2) * kKHalf + (k & 3) * 32) >> 4;
+                        tc_mma(tmem_s, q_lo + qoff, k_lo + koff, idesc, k > 0);
                     }
                     tc_commit(&misc->k_empty[ks]);
                     tc_commit(&misc->s_full[x]);
@@ -423,10 +421,15 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     if (ok) mbar_arrive(&misc->q_empty[qb]);             // no tile for this stream
                 } else {
                     if (ok) ok = issue_qk(x);
+                    const uint32_t idesc_pv = make_idesc(D, 1);
+                    const uint32_t p_lo = desc_lo_kmajor(p_addr);
                     for (int j = x; j < nt && ok; j += 2) {
                         if (j + 2 < nt) { ok = issue_qk(j + 2); if (!ok) break; }
                         const uint32_t vt = tiles + j;
                         const int vs = vt % C::NV;
+                        const uint32_t v_lo = desc_lo_mnmajor(smem_u32(smem + C::OFF_V)) + vs * (C::KV_BYTES >> 4);
+                        const int nk = cols16(j);
+                        const uint32_t acc0 = j >= 2;
                         ok = mbar_wait(&misc->p_full[x], pc & 1, misc);
                         if (!ok) break;
                         ok = mbar_wait(&misc->v_full[vs], (vt / C::NV) & 1, misc);
@@ -436,11 +439,9 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                             if (!ok) break;
                         }
                         tc_fence_after();
-                        const uint32_t idesc = make_idesc(D, 1);
-                        const uint32_t v_addr = smem_u32(smem + C::OFF_V + vs * C::KV_BYTES);
-                        const int nk = (tile_cols(u, j) + 15) >> 4;
-                        for (int k = 0; k < nk; ++k)
-                            tc_mma(tmem_o, desc_kmajor(p_addr + k * 32), desc_mnmajor(v_addr + k * 2048), idesc, (j >= 2 || k > 0));
+#pragma unroll
+                        for (int k = 0; k < kN / 16; ++k)
+                            if (k < nk) tc_mma(tmem_o, p_lo + k * 2, v_lo + k * 128, idesc_pv, k > 0 ? 1u : acc0);
                         tc_commit(&misc->v_empty[vs]);
                         tc_commit(&misc->p_empty[x]);
                         if (j + 2 >= nt) tc_commit(&misc->o_full[x]);
