@@ -48,6 +48,7 @@ constexpr uint32_t kColS = 0, kColO = 128;
 constexpr int kRegsIo = 80, kRegsSoftmax = 208;
 constexpr int kBoxKinds = 4;               // suffix boxes of 4, 8, 12, 16 cache rows
 constexpr int kPad = 4;                    // a branch's cached tokens occupy a multiple of 4 packed columns
+constexpr int kQAfter = 1;                 // the Q tile is loaded after K tiles 0..kQAfter of its unit
 constexpr int kRounds = 4;                 // a unit has at most 128 branches: 4 rounds of 32 lanes
 constexpr int kConsumerWarps = 11;         // warps that read unit descriptors (all but the scheduler)
 
@@ -58,8 +59,9 @@ template <int D> struct Cfg {
     static constexpr int NK = D == 128 ? 4 : 8;                  // K stages
     static constexpr int NV = D == 128 ? 4 : 8;                  // V stages
     static constexpr int OFF_Q = 0;
-    static constexpr int OFF_P = OFF_Q + 2 * Q_BYTES;
-    static constexpr int OFF_K = OFF_P + 2 * kPBytes;
+    static constexpr int NQ = D == 128 ? 1 : 2;                  // Q stages
+    static constexpr int OFF_P = OFF_Q + NQ * Q_BYTES;
+    static constexpr int OFF_K = OFF_P + 4 * kPBytes;           // two P tiles per stream
     static constexpr int OFF_V = OFF_K + NK * KV_BYTES;
     static constexpr int OFF_MISC = OFF_V + NV * KV_BYTES;
     static constexpr int SMEM = OFF_MISC + 3072;                 // + misc; the dynamic segment itself is 1024-B aligned
@@ -105,7 +107,7 @@ static_assert(sizeof(UnitDesc) == 48 + 4 * kM + 4 * kM, "descriptor size");
 struct Misc {
     unsigned long long q_full[2], q_empty[2];
     unsigned long long k_full[8], k_empty[8], v_full[8], v_empty[8];
-    unsigned long long s_full[2], s_empty[2], p_full[2], p_empty[2], o_full[2];
+    unsigned long long s_full[2], s_empty[2], p_full[4], p_empty[4], o_full[2];
     unsigned long long o_free, ml_full, desc_full[2], desc_empty[2];
     uint32_t tmem_base;
     int abort_flag;
@@ -257,9 +259,9 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         for (int i = 0; i < 2; ++i) {
             mbar_init(&misc->q_full[i], 1);  mbar_init(&misc->q_empty[i], 2);
             mbar_init(&misc->s_full[i], 1);  mbar_init(&misc->s_empty[i], 4);
-            mbar_init(&misc->p_full[i], 4);  mbar_init(&misc->p_empty[i], 1);
             mbar_init(&misc->o_full[i], 1);
         }
+        for (int i = 0; i < 4; ++i) { mbar_init(&misc->p_full[i], 4); mbar_init(&misc->p_empty[i], 1); }
         for (int i = 0; i < 8; ++i) {
             mbar_init(&misc->k_full[i], 1); mbar_init(&misc->k_empty[i], 1);
             mbar_init(&misc->v_full[i], 1); mbar_init(&misc->v_empty[i], 1);
@@ -301,15 +303,6 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             if (u.nt < 0) break;
             const int nt = u.nt;
             if (nt > 0) {
-                const int qb = qc & 1;
-                ok = mbar_wait_warp(&misc->q_empty[qb], ((qc >> 1) & 1) ^ 1, misc);
-                if (!ok) break;
-                if (lane == 0) {
-                    mbar_expect_tx(&misc->q_full[qb], C::Q_BYTES);
-                    for (int h = 0; h < C::HALVES; ++h)
-                        tma_load_4d(smem + C::OFF_Q + qb * C::Q_BYTES + h * kQHalf, &map_q, &misc->q_full[qb], h * 64, 0, u.head, u.row0);
-                }
-                ++qc;
                 // One tile: a prefix tile is two boxes issued by lane 0; a suffix tile is packed from one box per
                 // branch (and half), every lane placing the part of its branches that falls into the tile.  K boxes
                 // are 4, 8, 12 or 16 rows high and may read up to three rows past the branch's length (their columns
@@ -359,6 +352,19 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         fill(t, smem + C::OFF_K + ks * C::KV_BYTES, &misc->k_full[ks], map_k, smaps.k, false);
                         ++kc;
                     }
+                    if (t == min(kQAfter, nt - 1)) {
+                        // The Q tile is asked for after the unit's first K tiles: its buffer is released late in the
+                        // previous unit, and waiting for it first would hold up the tiles that can be fetched already.
+                        const int qb = qc % C::NQ;
+                        ok = mbar_wait_warp(&misc->q_empty[qb], ((qc / C::NQ) & 1) ^ 1, misc);
+                        if (!ok) break;
+                        if (lane == 0) {
+                            mbar_expect_tx(&misc->q_full[qb], C::Q_BYTES);
+                            for (int h = 0; h < C::HALVES; ++h)
+                                tma_load_4d(smem + C::OFF_Q + qb * C::Q_BYTES + h * kQHalf, &map_q, &misc->q_full[qb], h * 64, 0, u.head, u.row0);
+                        }
+                        ++qc;
+                    }
                     if (t >= 2) {
                         const int vs = vc % C::NV;
                         ok = mbar_wait_warp(&misc->v_empty[vs], ((vc / C::NV) & 1) ^ 1, misc);
@@ -378,7 +384,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             uint32_t qc = 0, tiles = 0;                   // units with tiles so far; tiles of earlier units
             uint32_t sc = 0, pc = 0;                      // this stream: S tiles issued, P tiles consumed
             bool ok = true;
-            const uint32_t p_addr = smem_u32(smem + C::OFF_P + x * kPBytes);
+            const uint32_t p_addr = smem_u32(smem + C::OFF_P + x * 2 * kPBytes);     // this stream's two P tiles
             const uint32_t tmem_s = tmem + kColS + x * kN, tmem_o = tmem + kColO + x * 128;
             for (uint32_t ui = 0; ok; ++ui) {
                 const int slot = ui & 1;
@@ -389,13 +395,13 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 if (u.nt < 0) break;
                 const int nt = u.nt;
                 if (nt == 0) continue;
-                const int qb = qc & 1;
+                const int qb = qc % C::NQ;
                 const uint32_t q_lo = desc_lo_kmajor(smem_u32(smem + C::OFF_Q + qb * C::Q_BYTES));
                 const int ns = nt - u.np;
                 // columns of tile j: only the last suffix tile and the last prefix tile can be partial
                 const int last_s = u.stot - (ns - 1) * kN, last_p = u.key_count - (u.np - 1) * kN;
                 auto cols16 = [&](int j) { return ((j == ns - 1 ? last_s : (j == nt - 1 ? last_p : kN)) + 15) >> 4; };
-                ok = mbar_wait(&misc->q_full[qb], (qc >> 1) & 1, misc);
+                ok = mbar_wait(&misc->q_full[qb], (qc / C::NQ) & 1, misc);
                 ++qc;
                 auto issue_qk = [&](int j) {
                     const uint32_t kt = tiles + j;
@@ -422,7 +428,6 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 } else {
                     if (ok) ok = issue_qk(x);
                     const uint32_t idesc_pv = make_idesc(D, 1);
-                    const uint32_t p_lo = desc_lo_kmajor(p_addr);
                     for (int j = x; j < nt && ok; j += 2) {
                         if (j + 2 < nt) { ok = issue_qk(j + 2); if (!ok) break; }
                         const uint32_t vt = tiles + j;
@@ -430,7 +435,9 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         const uint32_t v_lo = desc_lo_mnmajor(smem_u32(smem + C::OFF_V)) + vs * (C::KV_BYTES >> 4);
                         const int nk = cols16(j);
                         const uint32_t acc0 = j >= 2;
-                        ok = mbar_wait(&misc->p_full[x], pc & 1, misc);
+                        const int pb = x * 2 + (pc & 1);
+                        const uint32_t p_lo = desc_lo_kmajor(p_addr + (pc & 1) * kPBytes);
+                        ok = mbar_wait(&misc->p_full[pb], (pc >> 1) & 1, misc);
                         if (!ok) break;
                         ok = mbar_wait(&misc->v_full[vs], (vt / C::NV) & 1, misc);
                         if (!ok) break;
@@ -443,7 +450,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         for (int k = 0; k < kN / 16; ++k)
                             if (k < nk) tc_mma(tmem_o, p_lo + k * 2, v_lo + k * 128, idesc_pv, k > 0 ? 1u : acc0);
                         tc_commit(&misc->v_empty[vs]);
-                        tc_commit(&misc->p_empty[x]);
+                        tc_commit(&misc->p_empty[pb]);
                         if (j + 2 >= nt) tc_commit(&misc->o_full[x]);
                         ++pc;
                     }
@@ -564,12 +571,13 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const uint32_t lane_base = static_cast<uint32_t>(quad * 32) << 16;
         const uint32_t tmem_s = tmem + lane_base + kColS + x * kN;
         const uint32_t tmem_o = tmem + lane_base + kColO + x * 128;
-        uint8_t* p_tile = smem + C::OFF_P + x * kPBytes;
-        float2* ml_mine = reinterpret_cast<float2*>(p_tile);                          // (max, sum) exchange area
-        const float2* ml_a = reinterpret_cast<const float2*>(smem + C::OFF_P);
-        const float2* ml_b = reinterpret_cast<const float2*>(smem + C::OFF_P + kPBytes);
+        // Each stream owns two P tiles and alternates between them, so a new P tile is written while the tensor core
+        // still reads the previous one.  pw counts the P tiles this stream has written so far, pw_other those of the other stream (the groups keep both
+        // counts: the epilogue finds the other stream's (max, sum) area in that stream's next P tile).
+        uint8_t* p_base = smem + C::OFF_P + x * 2 * kPBytes;
         const int b_row = row / G;                       // branch of this row inside the unit
-        uint32_t s_cnt = 0, pe_cnt = 0;
+        uint32_t s_cnt = 0;
+        uint32_t pw = 0, pw_other = 0;
         uint32_t of_a = 0, of_b = 0;
         bool ok = true;
         for (uint32_t unit_idx = 0; ok; ++unit_idx) {
@@ -607,7 +615,6 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&misc->s_empty[x]);
 
-                bool waited = false;
                 if (warp_active) {
                     int lo = 0, hi;
                     const int ns = nt - u.np;
@@ -640,8 +647,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         const bool grow = !fresh && tmax > m + kRescaleSlack;
                         if (__any_sync(0xffffffffu, grow)) {
                             // O must be rescaled: wait until this stream's previous P V product has landed in TMEM
-                            ok = mbar_wait_warp(&misc->p_empty[x], pe_cnt & 1, misc);
-                            ++pe_cnt; waited = true;
+                            ok = mbar_wait_warp(&misc->p_empty[x * 2 + ((pw - 1) & 1)], ((pw - 1) >> 1) & 1, misc);
                             if (ok) {
                                 tc_fence_after();
                                 const float m_new = grow ? tmax : m;
@@ -662,15 +668,13 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         }
                     }
                 }
-                if (i > 0 && !waited) {
-                    ok = ok && mbar_wait_warp(&misc->p_empty[x], pe_cnt & 1, misc);   // previous P V has consumed the P tile
-                    ++pe_cnt;
-                }
+                const int pb = pw & 1;                 // the P V product that read this P tile two tiles ago is done
+                ok = ok && mbar_wait_warp(&misc->p_empty[x * 2 + pb], ((pw >> 1) & 1) ^ 1, misc);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 if (warp_active) {
                     const float neg_m = (m == -INFINITY) ? 0.f : -m;
-                    uint8_t* prow = p_tile + row * 128;
+                    uint8_t* prow = p_base + pb * kPBytes + row * 128;
                     float lsum[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                     for (int kc8 = 0; kc8 < kN / 8; ++kc8) {
@@ -690,17 +694,22 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&misc->p_full[x]);
+                if (lane == 0) mbar_arrive(&misc->p_full[x * 2 + pb]);
+                ++pw;
             }
             if (!ok) break;
 
             // ------------------------------------ epilogue ------------------------------------
             // both groups merge the two streams; group x writes output columns [x*D/2, (x+1)*D/2)
-            if (n_mine > 0) {                            // this stream's last P V has landed (and P is free)
-                ok = mbar_wait_warp(&misc->p_empty[x], pe_cnt & 1, misc);
-                ++pe_cnt;
-                if (!ok) break;
-            }
+            pw_other += (nt + x) >> 1;                 // tiles the other stream writes in this unit
+            // the stream's next P tile is idle until the next unit: it carries the (max, sum) exchange and the output staging
+            ok = mbar_wait_warp(&misc->p_empty[x * 2 + (pw & 1)], ((pw >> 1) & 1) ^ 1, misc);
+            if (!ok) break;
+            uint8_t* p_tile = p_base + (pw & 1) * kPBytes;
+            float2* ml_mine = reinterpret_cast<float2*>(p_tile);
+            const float2* ml_other = reinterpret_cast<const float2*>(smem + C::OFF_P + ((x ^ 1) * 2 + (pw_other & 1)) * kPBytes);
+            const float2* ml_a = x == 0 ? ml_mine : ml_other;
+            const float2* ml_b = x == 0 ? ml_other : ml_mine;
             ml_mine[row] = make_float2(m, l);
             __syncwarp();
             if (lane == 0) mbar_arrive(&misc->ml_full);
