@@ -237,6 +237,51 @@ __device__ __forceinline__ Unit read_unit(const UnitDesc& d) {
     return u;
 }
 
+// One K or V tile of a unit.  A prefix tile is two boxes issued by lane 0; a suffix tile is packed from one box per
+// branch (and half), every lane placing the part of its branches that falls into the tile.  K boxes are 4, 8, 12 or
+// 16 rows high and may read up to three rows past the branch's length (their columns are masked); V boxes (EXACT) have
+// the exact height, because whatever lies beyond a branch's length in the cache -- possibly NaN -- would otherwise be
+// multiplied by a zero probability.
+template <int D, bool EXACT>
+__device__ __forceinline__ void fill_tile(const Unit& u, int t, const int (&cs)[kRounds], const int (&len)[kRounds], const int (&off)[kRounds],
+                                          int lane, uint8_t* tile, unsigned long long* full, const CUtensorMap* pre, const CUtensorMap* suf)
+{
+    using C = Cfg<D>;
+    const int ns = u.nt - u.np;
+    if (t >= ns) {
+        if (lane == 0) {
+            mbar_expect_tx(full, C::KV_BYTES);
+            for (int h = 0; h < C::HALVES; ++h)
+                tma_load_3d(tile + h * kKHalf, pre, full, h * 64, u.head, u.kv_row0 + (t - ns) * kN);
+        }
+    } else {
+        const int c_lo = t * kN, c_hi = min(u.stot, c_lo + kN);
+        int rows_mine = 0;
+#pragma unroll
+        for (int r = 0; r < kRounds; ++r) {
+            const int plen = EXACT ? len[r] : (len[r] + kPad - 1) & ~(kPad - 1);
+            rows_mine += max(0, min(cs[r] + plen, c_hi) - max(cs[r], c_lo));
+        }
+        const int rows_all = __reduce_add_sync(0xffffffffu, rows_mine);
+        if (lane == 0) mbar_expect_tx(full, static_cast<uint32_t>(rows_all) * D * 2);
+#pragma unroll
+        for (int r = 0; r < kRounds; ++r) {
+            const int plen = EXACT ? len[r] : (len[r] + kPad - 1) & ~(kPad - 1);
+            const int lo = max(cs[r], c_lo), hi = min(cs[r] + plen, c_hi);
+            int n = hi - lo;
+            int row = off[r] + (lo - cs[r]);
+            int col = lo - c_lo;
+            while (n > 0) {
+                const int hb = min(n, 16);
+                const CUtensorMap* m = EXACT ? &suf[hb - 1] : &suf[hb / 4 - 1];
+                for (int h = 0; h < C::HALVES; ++h)
+                    tma_load_3d(tile + h * kKHalf + col * 128, m, full, h * 64, u.head, row);
+                row += hb; col += hb; n -= hb;
+            }
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------------------
@@ -285,9 +330,9 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&misc->tmem_base);
 
     if (warp == 0) {
-        // ======================================= TMA producer =======================================
+        // ================================ TMA producer of Q and K tiles ==============================
         reg_dealloc<kRegsIo>();
-        uint32_t qc = 0, kc = 0, vc = 0;
+        uint32_t qc = 0, kc = 0;
         bool ok = true;
         for (uint32_t ui = 0; ok; ++ui) {
             const int slot = ui & 1;
@@ -302,78 +347,26 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             if (lane == 0) mbar_arrive(&misc->desc_empty[slot]);
             if (u.nt < 0) break;
             const int nt = u.nt;
-            if (nt > 0) {
-                // One tile: a prefix tile is two boxes issued by lane 0; a suffix tile is packed from one box per
-                // branch (and half), every lane placing the part of its branches that falls into the tile.  K boxes
-                // are 4, 8, 12 or 16 rows high and may read up to three rows past the branch's length (their columns
-                // are masked); V boxes have the exact height, because whatever lies beyond a branch's length in the
-                // cache -- possibly NaN -- would otherwise be multiplied by a zero probability.
-                auto fill = [&](int t, uint8_t* tile, unsigned long long* full, const CUtensorMap& pre, const CUtensorMap* suf, bool exact) {
-                    const int ns = nt - u.np;
-                    if (t >= ns) {
-                        if (lane == 0) {
-                            mbar_expect_tx(full, C::KV_BYTES);
-                            for (int h = 0; h < C::HALVES; ++h)
-                                tma_load_3d(tile + h * kKHalf, &pre, full, h * 64, u.head, u.kv_row0 + (t - ns) * kN);
-                        }
-                    } else {
-                        const int c_lo = t * kN, c_hi = min(u.stot, c_lo + kN);
-                        int rows_mine = 0;
-#pragma unroll
-                        for (int r = 0; r < kRounds; ++r) {
-                            const int plen = exact ? len[r] : (len[r] + kPad - 1) & ~(kPad - 1);
-                            rows_mine += max(0, min(cs[r] + plen, c_hi) - max(cs[r], c_lo));
-                        }
-                        const int rows_all = __reduce_add_sync(0xffffffffu, rows_mine);
-                        if (lane == 0) mbar_expect_tx(full, static_cast<uint32_t>(rows_all) * D * 2);
-#pragma unroll
-                        for (int r = 0; r < kRounds; ++r) {
-                            const int plen = exact ? len[r] : (len[r] + kPad - 1) & ~(kPad - 1);
-                            const int lo = max(cs[r], c_lo), hi = min(cs[r] + plen, c_hi);
-                            int n = hi - lo;
-                            int row = off[r] + (lo - cs[r]);
-                            int col = lo - c_lo;
-                            while (n > 0) {
-                                const int hb = min(n, 16);
-                                const CUtensorMap* m = exact ? &suf[hb - 1] : &suf[hb / 4 - 1];
-                                for (int h = 0; h < C::HALVES; ++h)
-                                    tma_load_3d(tile + h * kKHalf + col * 128, m, full, h * 64, u.head, row);
-                                row += hb; col += hb; n -= hb;
-                            }
-                        }
+            for (int t = 0; t < nt && ok; ++t) {
+                const int ks = kc % C::NK;
+                ok = mbar_wait_warp(&misc->k_empty[ks], ((kc / C::NK) & 1) ^ 1, misc);
+                if (!ok) break;
+                fill_tile<D, false>(u, t, cs, len, off, lane, smem + C::OFF_K + ks * C::KV_BYTES, &misc->k_full[ks], &map_k, smaps.k);
+                ++kc;
+                if (t == min(kQAfter, nt - 1)) {
+                    // The Q tile is asked for after the unit's first K tiles: its buffer is released late in the
+                    // previous unit, and waiting for it first would hold up the tiles that can be fetched already.
+                    const int qb = qc % C::NQ;
+                    ok = mbar_wait_warp(&misc->q_empty[qb], ((qc / C::NQ) & 1) ^ 1, misc);
+                    if (!ok) break;
+                    if (lane == 0) {
+                        mbar_expect_tx(&misc->q_full[qb], C::Q_BYTES);
+                        for (int h = 0; h < C::HALVES; ++h)
+                            tma_load_4d(smem + C::OFF_Q + qb * C::Q_BYTES + h * kQHalf, &map_q, &misc->q_full[qb], h * 64, 0, u.head, u.row0);
                     }
-                };
-                // K runs two tiles ahead of V, the order in which the MMA warps consume them
-                for (int t = 0; t < nt + 2 && ok; ++t) {
-                    if (t < nt) {
-                        const int ks = kc % C::NK;
-                        ok = mbar_wait_warp(&misc->k_empty[ks], ((kc / C::NK) & 1) ^ 1, misc);
-                        if (!ok) break;
-                        fill(t, smem + C::OFF_K + ks * C::KV_BYTES, &misc->k_full[ks], map_k, smaps.k, false);
-                        ++kc;
-                    }
-                    if (t == min(kQAfter, nt - 1)) {
-                        // The Q tile is asked for after the unit's first K tiles: its buffer is released late in the
-                        // previous unit, and waiting for it first would hold up the tiles that can be fetched already.
-                        const int qb = qc % C::NQ;
-                        ok = mbar_wait_warp(&misc->q_empty[qb], ((qc / C::NQ) & 1) ^ 1, misc);
-                        if (!ok) break;
-                        if (lane == 0) {
-                            mbar_expect_tx(&misc->q_full[qb], C::Q_BYTES);
-                            for (int h = 0; h < C::HALVES; ++h)
-                                tma_load_4d(smem + C::OFF_Q + qb * C::Q_BYTES + h * kQHalf, &map_q, &misc->q_full[qb], h * 64, 0, u.head, u.row0);
-                        }
-                        ++qc;
-                    }
-                    if (t >= 2) {
-                        const int vs = vc % C::NV;
-                        ok = mbar_wait_warp(&misc->v_empty[vs], ((vc / C::NV) & 1) ^ 1, misc);
-                        if (!ok) break;
-                        fill(t - 2, smem + C::OFF_V + vs * C::KV_BYTES, &misc->v_full[vs], map_v, smaps.v, true);
-                        ++vc;
-                    }
-                    __syncwarp();
+                    ++qc;
                 }
+                __syncwarp();
             }
         }
     } else if (warp < 3) {
@@ -459,7 +452,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             }
         }
     } else if (warp < 4) {
-        // ========================================= scheduler ========================================
+        // ============================ scheduler and TMA producer of V tiles ==========================
         // Software pipeline over units, one stage per iteration, so that every global load is consumed an
         // iteration after it was issued: ticket (i+4) -> work item (i+3) -> document tables (i+2) ->
         // branch table (i+1) -> scan and publish (i).
@@ -468,6 +461,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const int Hkv = p.a.g.Hkv;
         const int64_t cache_rows = static_cast<int64_t>(p.a.n_slots) * p.a.g.suffix_cap;
         uint32_t* ticket = const_cast<uint32_t*>(&p.hdr->ticket);
+        uint32_t vc = 0;                                  // V tiles produced so far
         if (n_units == 0) {                              // nothing to do: publish the stop descriptor
             if (lane == 0) { misc->desc[0].nt = -1; mbar_arrive(&misc->desc_full[0]); }
         } else {
@@ -553,6 +547,22 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&misc->desc_full[slot]);
+            // ---- V tiles of the unit published one iteration ago (its descriptor slot is rewritten only after this) ----
+            if (ui >= 1) {
+                const UnitDesc& dv = misc->desc[slot ^ 1];
+                const Unit uv = read_unit(dv);
+                int vcs[kRounds], vlen[kRounds], voff[kRounds];
+#pragma unroll
+                for (int r = 0; r < kRounds; ++r) { vcs[r] = dv.cs[lane + 32 * r]; vlen[r] = dv.len[lane + 32 * r]; voff[r] = dv.off[lane + 32 * r]; }
+                for (int t = 0; t < uv.nt && ok; ++t) {
+                    const int vs = vc % C::NV;
+                    ok = mbar_wait_warp(&misc->v_empty[vs], ((vc / C::NV) & 1) ^ 1, misc);
+                    if (!ok) break;
+                    fill_tile<D, true>(uv, t, vcs, vlen, voff, lane, smem + C::OFF_V + vs * C::KV_BYTES, &misc->v_full[vs], &map_v, smaps.v);
+                    ++vc;
+                    __syncwarp();
+                }
+            }
             if (!live) break;
             // ---- shift the pipeline ----
             w0 = w1; w1 = w2; w2 = w3; w3 = w4; w4 = w5;
