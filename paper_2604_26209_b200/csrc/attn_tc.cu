@@ -205,6 +205,11 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
@@ -586,6 +591,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         // counts: the epilogue finds the other stream's (max, sum) area in that stream's next P tile).
         uint8_t* p_base = smem + C::OFF_P + x * 2 * kPBytes;
         const int b_row = row / G;                       // branch of this row inside the unit
+        const uint32_t g_magic = 0xFFFFFFFFu / static_cast<uint32_t>(G) + 1u;   // floor(r / G) = umulhi(r, g_magic) for r < 2^16, G > 1
         uint32_t s_cnt = 0;
         uint32_t pw = 0, pw_other = 0;
         uint32_t of_a = 0, of_b = 0;
@@ -612,21 +618,10 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             float m = -INFINITY, l = 0.f;
             for (int i = 0; i < n_mine && ok; ++i) {
                 const int j = x + 2 * i;
-                ok = mbar_wait_warp(&misc->s_full[x], s_cnt & 1, misc);
-                if (!ok) break;
-                ++s_cnt;
-                tc_fence_after();
-                uint32_t sv[kN];
+                // Columns of this tile the row may see.  A suffix tile holds a few branches each; a warp whose rows see
+                // none of them (known from the descriptor alone) skips the tile's scores and writes zero probabilities.
+                int lo = 0, hi = 0;
                 if (warp_active) {
-                    tmem_ld32(tmem_s, sv); tmem_ld32(tmem_s + 32, sv + 32);
-                    tmem_ld_wait();
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&misc->s_empty[x]);
-
-                if (warp_active) {
-                    int lo = 0, hi;
                     const int ns = nt - u.np;
                     if (j >= ns) {
                         hi = min(kN, u.key_count - (j - ns) * kN);
@@ -636,6 +631,22 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         hi = min(kN, my_cs + my_len - base);
                         if (hi < lo) hi = lo;
                     }
+                }
+                const bool vis = __any_sync(0xffffffffu, hi > lo);
+                ok = mbar_wait_warp(&misc->s_full[x], s_cnt & 1, misc);
+                if (!ok) break;
+                ++s_cnt;
+                tc_fence_after();
+                uint32_t sv[kN];
+                if (vis) {
+                    tmem_ld32(tmem_s, sv); tmem_ld32(tmem_s + 32, sv + 32);
+                    tmem_ld_wait();
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&misc->s_empty[x]);
+
+                if (vis) {
                     if (!__all_sync(0xffffffffu, lo == 0 && hi == kN)) {
                         const unsigned span = static_cast<unsigned>(hi - lo);
 #pragma unroll
@@ -644,10 +655,12 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     }
                     float t8[8];
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) t8[c] = __uint_as_float(sv[c]);
+                    for (int c = 0; c < 8; ++c) t8[c] = fmaxf(__uint_as_float(sv[c]), __uint_as_float(sv[c + 8]));
 #pragma unroll
-                    for (int c = 8; c < kN; ++c) t8[c & 7] = fmaxf(t8[c & 7], __uint_as_float(sv[c]));
-                    float tmax = fmaxf(fmaxf(fmaxf(t8[0], t8[1]), fmaxf(t8[2], t8[3])), fmaxf(fmaxf(t8[4], t8[5]), fmaxf(t8[6], t8[7])));
+                    for (int c = 16; c < kN; c += 16)
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) t8[k] = fmax3(t8[k], __uint_as_float(sv[c + k]), __uint_as_float(sv[c + 8 + k]));
+                    float tmax = fmax3(fmax3(t8[0], t8[1], t8[2]), fmax3(t8[3], t8[4], t8[5]), fmaxf(t8[6], t8[7]));
                     tmax *= p.scale_log2;
                     if (i == 0) {
                         m = tmax;
@@ -682,7 +695,12 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 ok = ok && mbar_wait_warp(&misc->p_empty[x * 2 + pb], ((pw >> 1) & 1) ^ 1, misc);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                if (warp_active) {
+                if (warp_active && !vis) {              // nothing visible for any row of the warp: P rows of zeros
+                    uint8_t* prow = p_base + pb * kPBytes + row * 128;
+#pragma unroll
+                    for (int kc8 = 0; kc8 < kN / 8; ++kc8) *reinterpret_cast<uint4*>(prow + (kc8 << 4)) = make_uint4(0, 0, 0, 0);
+                    fence_async_smem();
+                } else if (warp_active) {
                     const float neg_m = (m == -INFINITY) ? 0.f : -m;
                     uint8_t* prow = p_base + pb * kPBytes + row * 128;
                     float lsum[4] = {0.f, 0.f, 0.f, 0.f};
@@ -752,18 +770,19 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 #pragma unroll
                 for (int c = 0; c < 32; ++c) acc[c] = 0.f;
                 if (warp_active) {
-                    uint32_t ov[32];
-                    if (n_a > 0) {
+                    if (n_a > 0 && n_b > 0) {            // both streams: the two loads are in flight together
+                        uint32_t oa[32], ob[32];
+                        tmem_ld32(tmem + lane_base + kColO + x * HC + c0, oa);
+                        tmem_ld32(tmem + lane_base + kColO + 128 + x * HC + c0, ob);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) acc[c] = fmaf(cb, __uint_as_float(ob[c]), ca * __uint_as_float(oa[c]));
+                    } else if (n_a > 0) {
+                        uint32_t ov[32];
                         tmem_ld32(tmem + lane_base + kColO + x * HC + c0, ov);
                         tmem_ld_wait();
 #pragma unroll
                         for (int c = 0; c < 32; ++c) acc[c] = ca * __uint_as_float(ov[c]);
-                    }
-                    if (n_b > 0) {
-                        tmem_ld32(tmem + lane_base + kColO + 128 + x * HC + c0, ov);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) acc[c] = fmaf(cb, __uint_as_float(ov[c]), acc[c]);
                     }
                 }
                 if (c0 + 32 >= HC) {                     // all TMEM reads of this unit are done
@@ -790,7 +809,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         const int rl = 8 * i + (lane >> 2), ch = lane & 3;       // row inside the warp's 32, 16-byte piece
                         const uint4 pk = *reinterpret_cast<const uint4*>(stg + rl * 64 + (((ch ^ (rl >> 1)) & 3) << 4));
                         const int trow = quad * 32 + rl;
-                        const int tb = trow / G, tg = trow - tb * G;
+                        const int tb = G == 1 ? trow : static_cast<int>(__umulhi(static_cast<uint32_t>(trow), g_magic)), tg = trow - tb * G;
                         const int grow = u.row0 + tb;
                         if (trow < nrows && grow < p.a.max_rows)
                             *reinterpret_cast<uint4*>(p.a.o + (static_cast<int64_t>(grow) * p.a.g.Hq + u.head * G + tg) * D + x * HC + c0 + ch * 8) = pk;
