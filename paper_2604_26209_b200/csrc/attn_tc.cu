@@ -3,17 +3,19 @@
 // One persistent CTA per SM walks the step's work units.  A unit = (work item, kv head): up to
 // 128/G branches of one document (rows = branches x G query heads, the M dimension) against a chunk
 // of that document's prefix, so each prefix K/V byte is read from HBM once for all of the document's
-// branches.  Keys are consumed in tiles of 64: first the prefix tiles, then tiles into which the
-// branches' own cached tokens ("suffix") are packed back to back, each branch padded to a multiple of
-// four columns so that one TMA box of 4..16 cache rows places it (the few rows read beyond a branch's
-// length are masked); those tiles are masked block-diagonally (a row sees only its own branch's columns).  Even tiles
-// form stream A, odd tiles stream B, each with its own MMA-issuing warp, softmax group, score
-// buffer, probability tile and output accumulator, so the two streams run as independent
+// branches.  Keys are consumed in tiles of 64: first the tiles into which the branches' own cached
+// tokens ("suffix") are packed back to back, each branch padded to a multiple of four columns so
+// that one TMA box of 4..16 cache rows places it (the few K rows read beyond a branch's length are
+// masked; V boxes have the exact height), masked block-diagonally (a row sees only its own branch's
+// columns); then the prefix tiles.  The suffix tiles come first because their many small copies are
+// slow to issue and can be issued while the previous unit is still in its epilogue.  Even tiles form
+// stream A, odd tiles stream B, each with its own MMA-issuing warp, softmax group, score buffer,
+// pair of probability tiles and output accumulator, so the two streams run as independent
 // online-softmax pipelines over one K/V stream (a split-KV inside the CTA); the epilogue merges them.
 //
-//   warp 0        TMA producer: Q tile (double buffered), prefix K/V tiles (lane 0), suffix boxes (all lanes)
+//   warp 0        TMA producer of the Q tile and the K tiles (prefix: lane 0; suffix boxes: all lanes)
 //   warps 1-2     MMA issuers of streams A and B: S = Q K^T and O += P V (tcgen05.mma, TMEM accumulators)
-//   warp 3        idle (it completes the first warpgroup, which gives its registers away)
+//   warp 3        scheduler (draws units, publishes their descriptors) and TMA producer of the V tiles
 //   warps 4-7     softmax A     one thread per row: S from TMEM, online max/sum, P (bf16) to shared
 //   warps 8-11    softmax B     memory, rare rescale of O in TMEM; both groups share the epilogue
 //
@@ -460,7 +462,9 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         // ============================ scheduler and TMA producer of V tiles ==========================
         // Software pipeline over units, one stage per iteration, so that every global load is consumed an
         // iteration after it was issued: ticket (i+4) -> work item (i+3) -> document tables (i+2) ->
-        // branch table (i+1) -> scan and publish (i).
+        // branch table (i+1) -> scan and publish (i).  After publishing unit i the warp issues the V tiles of unit
+        // i-1: V is needed two tiles later than K, and two issuing warps keep up with the many small copies of the
+        // suffix tiles where one did not.
         reg_dealloc<kRegsIo>();
         const int n_units = p.hdr->n_work * p.a.g.Hkv;
         const int Hkv = p.a.g.Hkv;
