@@ -43,6 +43,9 @@ STRUCTS = {
     "one_group_96": lambda: synth.config_custom("wide", Hq=32, Hkv=8, D=128, theta=500000.0, cap=8,
                                                 prefix_lens=[700], branch_cnts=[96], depth_hi=8, seed=6),
     "few_alive": lambda: _ragged(7, alive_frac=0.1),
+    # one query head per kv head: 128 branches per unit, four rounds of branch tables, dozens of suffix tiles per unit
+    "g1_many_branches": lambda: synth.config_custom("g1", Hq=2, Hkv=2, D=128, theta=10000.0, cap=32,
+                                                    prefix_lens=[200, 50, 0], branch_cnts=[200, 130, 70], depth_hi=32, seed=9),
     "long_small": lambda: synth.config_custom("long", Hq=32, Hkv=8, D=128, theta=500000.0, cap=32,
                                               prefix_lens=[4096, 1025, 3000], branch_cnts=[12, 12, 12], depth_hi=32, seed=8),
 }
