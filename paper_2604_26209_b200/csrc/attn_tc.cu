@@ -47,26 +47,29 @@ constexpr float kRescaleSlack = 8.0f;      // tolerated growth of the row maximu
 constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz
 constexpr uint32_t kColS = 0, kColO = 128;
 // registers per thread after the warpgroups have traded them (3 x 128 threads, 168 each at launch)
-constexpr int kRegsIo = 80, kRegsSoftmax = 208;
+constexpr int kRegsIo = 96, kRegsSoftmax = 200;
+// setmaxnreg only moves registers inside the CTA's own allocation (168 x 384 threads at launch): a request beyond
+// that pool would block forever
+static_assert(kRegsIo + 2 * kRegsSoftmax <= 3 * 168, "registers traded between the warpgroups exceed the CTA's allocation");
 constexpr int kBoxKinds = 4;               // suffix boxes of 4, 8, 12, 16 cache rows
 constexpr int kPad = 4;                    // a branch's cached tokens occupy a multiple of 4 packed columns
-constexpr int kQAfter = 1;                 // the Q tile is loaded after K tiles 0..kQAfter of its unit
 constexpr int kRounds = 4;                 // a unit has at most 128 branches: 4 rounds of 32 lanes
-constexpr int kConsumerWarps = 11;         // warps that read unit descriptors (all but the scheduler)
+constexpr int kDescReaders = 5;            // readers of a pipeline's unit descriptor: its MMA thread and its four softmax warps
+constexpr int kMaxStages = 4;              // K or V stages of one pipeline (barrier storage)
 
 template <int D> struct Cfg {
     static constexpr int HALVES = D / 64;
     static constexpr int Q_BYTES = HALVES * kQHalf;
     static constexpr int KV_BYTES = HALVES * kKHalf;            // one K or V tile
-    static constexpr int NK = D == 128 ? 4 : 8;                  // K stages
-    static constexpr int NV = D == 128 ? 4 : 8;                  // V stages
-    static constexpr int OFF_Q = 0;
-    static constexpr int NQ = D == 128 ? 1 : 2;                  // Q stages
-    static constexpr int OFF_P = OFF_Q + NQ * Q_BYTES;
-    static constexpr int OFF_K = OFF_P + 4 * kPBytes;           // two P tiles per stream
-    static constexpr int OFF_V = OFF_K + NK * KV_BYTES;
-    static constexpr int OFF_MISC = OFF_V + NV * KV_BYTES;
+    static constexpr int NK = D == 128 ? 2 : 4;                  // K stages of each pipeline
+    static constexpr int NV = D == 128 ? 2 : 4;                  // V stages of each pipeline
+    static constexpr int OFF_Q = 0;                              // one Q tile per pipeline
+    static constexpr int OFF_P = OFF_Q + 2 * Q_BYTES;           // one P tile per pipeline
+    static constexpr int OFF_K = OFF_P + 2 * kPBytes;
+    static constexpr int OFF_V = OFF_K + 2 * NK * KV_BYTES;
+    static constexpr int OFF_MISC = OFF_V + 2 * NV * KV_BYTES;
     static constexpr int SMEM = OFF_MISC + 3072;                 // + misc; the dynamic segment itself is 1024-B aligned
+    static_assert(NK <= kMaxStages && NV <= kMaxStages, "barrier storage");
 };
 static_assert(Cfg<128>::SMEM <= 232448, "shared memory budget");
 
@@ -102,19 +105,18 @@ struct UnitDesc {
     int pad[2];
     uint16_t cs[kM];     // per branch: packed column of its first cached token
     uint16_t len[kM];    // per branch: cached tokens visible (0 for a bad table entry)
-    int off[kM];         // per branch: first cache row
 };
-static_assert(sizeof(UnitDesc) == 48 + 4 * kM + 4 * kM, "descriptor size");
+static_assert(sizeof(UnitDesc) == 48 + 4 * kM, "descriptor size");
 
 struct Misc {
     unsigned long long q_full[2], q_empty[2];
-    unsigned long long k_full[8], k_empty[8], v_full[8], v_empty[8];
-    unsigned long long s_full[2], s_empty[2], p_full[4], p_empty[4], o_full[2];
-    unsigned long long o_free, ml_full, desc_full[2], desc_empty[2];
+    unsigned long long k_full[2][kMaxStages], k_empty[2][kMaxStages], v_full[2][kMaxStages], v_empty[2][kMaxStages];
+    unsigned long long s_full[2], s_empty[2], p_full[2], p_empty[2], o_full[2], o_free[2];
+    unsigned long long desc_full[2], desc_empty[2];
     uint32_t tmem_base;
     int abort_flag;
     int pad[2];
-    UnitDesc desc[2];
+    UnitDesc desc[2];    // one per pipeline
 };
 
 static_assert(sizeof(Misc) <= 3072, "misc block");
@@ -309,17 +311,16 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < 2; ++i) {
-            mbar_init(&misc->q_full[i], 1);  mbar_init(&misc->q_empty[i], 2);
+            mbar_init(&misc->q_full[i], 1);  mbar_init(&misc->q_empty[i], 1);
             mbar_init(&misc->s_full[i], 1);  mbar_init(&misc->s_empty[i], 4);
-            mbar_init(&misc->o_full[i], 1);
+            mbar_init(&misc->p_full[i], 4);  mbar_init(&misc->p_empty[i], 1);
+            mbar_init(&misc->o_full[i], 1);  mbar_init(&misc->o_free[i], 4);
+            mbar_init(&misc->desc_full[i], 1); mbar_init(&misc->desc_empty[i], kDescReaders);
+            for (int k = 0; k < kMaxStages; ++k) {
+                mbar_init(&misc->k_full[i][k], 1); mbar_init(&misc->k_empty[i][k], 1);
+                mbar_init(&misc->v_full[i][k], 1); mbar_init(&misc->v_empty[i][k], 1);
+            }
         }
-        for (int i = 0; i < 4; ++i) { mbar_init(&misc->p_full[i], 4); mbar_init(&misc->p_empty[i], 1); }
-        for (int i = 0; i < 8; ++i) {
-            mbar_init(&misc->k_full[i], 1); mbar_init(&misc->k_empty[i], 1);
-            mbar_init(&misc->v_full[i], 1); mbar_init(&misc->v_empty[i], 1);
-        }
-        mbar_init(&misc->o_free, 8); mbar_init(&misc->ml_full, 8);
-        for (int i = 0; i < 2; ++i) { mbar_init(&misc->desc_full[i], 1); mbar_init(&misc->desc_empty[i], kConsumerWarps); }
         misc->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -336,162 +337,45 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&misc->tmem_base);
 
-    if (warp == 0) {
-        // ================================ TMA producer of Q and K tiles ==============================
+    if (warp == 0 || warp == 3) {
+        // ============================ scheduler and TMA producer of one pipeline =====================
+        // Software pipeline over the pipeline's units, one stage per iteration, so that every global load is
+        // consumed an iteration after it was issued: ticket (i+4) -> work item (i+3) -> document tables (i+2) ->
+        // branch table (i+1) -> scan, publish and produce the tiles (i).  (An iteration lasts a whole unit, ten
+        // microseconds or more, so one stage per iteration is ample for an L2 round trip.)
         reg_dealloc<kRegsIo>();
-        uint32_t qc = 0, kc = 0;
-        bool ok = true;
-        for (uint32_t ui = 0; ok; ++ui) {
-            const int slot = ui & 1;
-            ok = mbar_wait_warp(&misc->desc_full[slot], (ui >> 1) & 1, misc);
-            if (!ok) break;
-            const UnitDesc& d = misc->desc[slot];
-            const Unit u = read_unit(d);
-            int cs[kRounds], len[kRounds], off[kRounds];
-#pragma unroll
-            for (int r = 0; r < kRounds; ++r) { cs[r] = d.cs[lane + 32 * r]; len[r] = d.len[lane + 32 * r]; off[r] = d.off[lane + 32 * r]; }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&misc->desc_empty[slot]);
-            if (u.nt < 0) break;
-            const int nt = u.nt;
-            for (int t = 0; t < nt && ok; ++t) {
-                const int ks = kc % C::NK;
-                ok = mbar_wait_warp(&misc->k_empty[ks], ((kc / C::NK) & 1) ^ 1, misc);
-                if (!ok) break;
-                fill_tile<D, false>(u, t, cs, len, off, lane, smem + C::OFF_K + ks * C::KV_BYTES, &misc->k_full[ks], &map_k, smaps.k);
-                ++kc;
-                if (t == min(kQAfter, nt - 1)) {
-                    // The Q tile is asked for after the unit's first K tiles: its buffer is released late in the
-                    // previous unit, and waiting for it first would hold up the tiles that can be fetched already.
-                    const int qb = qc % C::NQ;
-                    ok = mbar_wait_warp(&misc->q_empty[qb], ((qc / C::NQ) & 1) ^ 1, misc);
-                    if (!ok) break;
-                    if (lane == 0) {
-                        mbar_expect_tx(&misc->q_full[qb], C::Q_BYTES);
-                        for (int h = 0; h < C::HALVES; ++h)
-                            tma_load_4d(smem + C::OFF_Q + qb * C::Q_BYTES + h * kQHalf, &map_q, &misc->q_full[qb], h * 64, 0, u.head, u.row0);
-                    }
-                    ++qc;
-                }
-                __syncwarp();
-            }
-        }
-    } else if (warp < 3) {
-        // ================================ MMA issuers (one per stream) ===============================
-        reg_dealloc<kRegsIo>();
-        if (lane == 0) {
-            const int x = warp - 1;                      // stream: tiles x, x+2, ...
-            uint32_t qc = 0, tiles = 0;                   // units with tiles so far; tiles of earlier units
-            uint32_t sc = 0, pc = 0;                      // this stream: S tiles issued, P tiles consumed
-            bool ok = true;
-            const uint32_t p_addr = smem_u32(smem + C::OFF_P + x * 2 * kPBytes);     // this stream's two P tiles
-            const uint32_t tmem_s = tmem + kColS + x * kN, tmem_o = tmem + kColO + x * 128;
-            for (uint32_t ui = 0; ok; ++ui) {
-                const int slot = ui & 1;
-                ok = mbar_wait(&misc->desc_full[slot], (ui >> 1) & 1, misc);
-                if (!ok) break;
-                const Unit u = read_unit(misc->desc[slot]);
-                mbar_arrive(&misc->desc_empty[slot]);
-                if (u.nt < 0) break;
-                const int nt = u.nt;
-                if (nt == 0) continue;
-                const int qb = qc % C::NQ;
-                const uint32_t q_lo = desc_lo_kmajor(smem_u32(smem + C::OFF_Q + qb * C::Q_BYTES));
-                const int ns = nt - u.np;
-                // columns of tile j: only the last suffix tile and the last prefix tile can be partial
-                const int last_s = u.stot - (ns - 1) * kN, last_p = u.key_count - (u.np - 1) * kN;
-                auto cols16 = [&](int j) { return ((j == ns - 1 ? last_s : (j == nt - 1 ? last_p : kN)) + 15) >> 4; };
-                ok = mbar_wait(&misc->q_full[qb], (qc / C::NQ) & 1, misc);
-                ++qc;
-                auto issue_qk = [&](int j) {
-                    const uint32_t kt = tiles + j;
-                    const int ks = kt % C::NK;
-                    const uint32_t idesc = make_idesc(cols16(j) << 4, 0);
-                    const uint32_t k_lo = desc_lo_kmajor(smem_u32(smem + C::OFF_K)) + ks * (C::KV_BYTES >> 4);
-                    if (!mbar_wait(&misc->k_full[ks], (kt / C::NK) & 1, misc)) return false;
-                    if (!mbar_wait(&misc->s_empty[x], (sc & 1) ^ 1, misc)) return false;
-                    tc_fence_after();
-#pragma unroll
-                    for (int k = 0; k < D / 16; ++k) {
-                        const uint32_t qoff = ((k >> 2) * kQHalf + (k & 3) * 32) >> 4;
-                        const uint32_t koff = ((k >> 2) * kKHalf + (k & 3) * 32) >> 4;
-                        tc_mma(tmem_s, q_lo + qoff, k_lo + koff, idesc, k > 0);
-                    }
-                    tc_commit(&misc->k_empty[ks]);
-                    tc_commit(&misc->s_full[x]);
-                    if (j + 2 >= nt) tc_commit(&misc->q_empty[qb]);     // this stream's last use of the Q tile
-                    ++sc;
-                    return true;
-                };
-                if (x >= nt) {
-                    if (ok) mbar_arrive(&misc->q_empty[qb]);             // no tile for this stream
-                } else {
-                    if (ok) ok = issue_qk(x);
-                    const uint32_t idesc_pv = make_idesc(D, 1);
-                    for (int j = x; j < nt && ok; j += 2) {
-                        if (j + 2 < nt) { ok = issue_qk(j + 2); if (!ok) break; }
-                        const uint32_t vt = tiles + j;
-                        const int vs = vt % C::NV;
-                        const uint32_t v_lo = desc_lo_mnmajor(smem_u32(smem + C::OFF_V)) + vs * (C::KV_BYTES >> 4);
-                        const int nk = cols16(j);
-                        const uint32_t acc0 = j >= 2;
-                        const int pb = x * 2 + (pc & 1);
-                        const uint32_t p_lo = desc_lo_kmajor(p_addr + (pc & 1) * kPBytes);
-                        ok = mbar_wait(&misc->p_full[pb], (pc >> 1) & 1, misc);
-                        if (!ok) break;
-                        ok = mbar_wait(&misc->v_full[vs], (vt / C::NV) & 1, misc);
-                        if (!ok) break;
-                        if (j < 2 && ui > 0) {                // the previous unit's epilogue has read O
-                            ok = mbar_wait(&misc->o_free, (ui - 1) & 1, misc);
-                            if (!ok) break;
-                        }
-                        tc_fence_after();
-#pragma unroll
-                        for (int k = 0; k < kN / 16; ++k)
-                            if (k < nk) tc_mma(tmem_o, p_lo + k * 2, v_lo + k * 128, idesc_pv, k > 0 ? 1u : acc0);
-                        tc_commit(&misc->v_empty[vs]);
-                        tc_commit(&misc->p_empty[pb]);
-                        if (j + 2 >= nt) tc_commit(&misc->o_full[x]);
-                        ++pc;
-                    }
-                }
-                tiles += nt;
-            }
-        }
-    } else if (warp < 4) {
-        // ============================ scheduler and TMA producer of V tiles ==========================
-        // Software pipeline over units, one stage per iteration, so that every global load is consumed an
-        // iteration after it was issued: ticket (i+4) -> work item (i+3) -> document tables (i+2) ->
-        // branch table (i+1) -> scan and publish (i).  After publishing unit i the warp issues the V tiles of unit
-        // i-1: V is needed two tiles later than K, and two issuing warps keep up with the many small copies of the
-        // suffix tiles where one did not.
-        reg_dealloc<kRegsIo>();
+        const int x = warp == 0 ? 0 : 1;
         const int n_units = p.hdr->n_work * p.a.g.Hkv;
         const int Hkv = p.a.g.Hkv;
         const int64_t cache_rows = static_cast<int64_t>(p.a.n_slots) * p.a.g.suffix_cap;
         uint32_t* ticket = const_cast<uint32_t*>(&p.hdr->ticket);
-        uint32_t vc = 0;                                  // V tiles produced so far
+        UnitDesc& d = misc->desc[x];
+        uint8_t* k_ring = smem + C::OFF_K + x * C::NK * C::KV_BYTES;
+        uint8_t* v_ring = smem + C::OFF_V + x * C::NV * C::KV_BYTES;
+        uint8_t* q_tile = smem + C::OFF_Q + x * C::Q_BYTES;
         if (n_units == 0) {                              // nothing to do: publish the stop descriptor
-            if (lane == 0) { misc->desc[0].nt = -1; mbar_arrive(&misc->desc_full[0]); }
+            if (lane == 0) { d.nt = -1; mbar_arrive(&misc->desc_full[x]); }
         } else {
-        // The first five units of a CTA are fixed (unit = CTA + i * grid), which fills the pipeline without a
-        // chain of atomics; later units are drawn from the step's ticket counter, so faster SMs take more.
+        // The first units of a pipeline are fixed (unit = 2 * CTA + pipeline + i * 2 * grid), which fills the software
+        // pipeline without a chain of atomics; later units are drawn from the step's ticket counter, so faster SMs
+        // (and the pipeline that got shorter units) take more.
         constexpr int kStatic = 5;
-        const uint32_t first_dynamic = static_cast<uint32_t>(kStatic) * gridDim.x;
-        auto draw = [&]() {                              // next unit index of this CTA (lane 0 draws, all lanes get it)
+        const uint32_t first_dynamic = static_cast<uint32_t>(kStatic) * 2u * gridDim.x;
+        auto draw = [&]() {                              // next unit index (lane 0 draws, all lanes get it)
             uint32_t t = 0;
             if (lane == 0) t = atomicAdd(ticket, 1u);
             t = __shfl_sync(0xffffffffu, t, 0);
             return static_cast<int>(min(t + first_dynamic, static_cast<uint32_t>(n_units)));
         };
-        auto fixed = [&](int i) { return static_cast<int>(min(blockIdx.x + static_cast<uint32_t>(i) * gridDim.x, static_cast<uint32_t>(n_units))); };
-        int w0 = fixed(0), w1 = fixed(1), w2 = fixed(2), w3 = fixed(3), w4 = fixed(4);
+        auto fixed = [&](int i) {
+            return static_cast<int>(min(2u * blockIdx.x + static_cast<uint32_t>(x) + static_cast<uint32_t>(i) * 2u * gridDim.x, static_cast<uint32_t>(n_units)));
+        };
+        int w0 = fixed(0), w1 = fixed(1), w2 = fixed(2), w3 = fixed(3);
         auto item_of = [&](int w) { return p.work[min(w, max(n_units - 1, 0)) / Hkv]; };
-        WorkItem it3 = item_of(w3), it2 = item_of(w2), it1 = item_of(w1), it0 = item_of(w0);
-        int das2 = p.a.doc_active_start[it2.doc], dks2 = p.a.doc_kv_start[it2.doc];
+        WorkItem it2 = item_of(w2), it1 = item_of(w1), it0 = item_of(w0);
         int das1 = p.a.doc_active_start[it1.doc], dks1 = p.a.doc_kv_start[it1.doc];
         int das0 = p.a.doc_active_start[it0.doc], dks0 = p.a.doc_kv_start[it0.doc];
-        int rl1[kRounds], ro1[kRounds], rl0[kRounds], ro0[kRounds];            // raw branch tables of units i+1 and i
+        int rl0[kRounds], ro0[kRounds];                                        // raw branch table of unit i
         auto load_tab = [&](int w, const WorkItem& it, int das, int* rl, int* ro) {
 #pragma unroll
             for (int r = 0; r < kRounds; ++r) {
@@ -504,24 +388,23 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 }
             }
         };
-        load_tab(w1, it1, das1, rl1, ro1);
         load_tab(w0, it0, das0, rl0, ro0);
+        uint32_t qc = 0, kc = 0, vc = 0;
         bool ok = true;
         for (uint32_t ui = 0; ok; ++ui) {
             // ---- issue the next stage of every unit in flight (results are used in the next iteration) ----
-            const int w5 = draw();
-            const WorkItem it4 = item_of(w4);
-            const int das3 = p.a.doc_active_start[it3.doc], dks3 = p.a.doc_kv_start[it3.doc];
-            int rl2[kRounds], ro2[kRounds];
-            load_tab(w2, it2, das2, rl2, ro2);
+            const int w4 = ui == 0 ? fixed(4) : draw();
+            const WorkItem it3 = item_of(w3);
+            const int das2 = p.a.doc_active_start[it2.doc], dks2 = p.a.doc_kv_start[it2.doc];
+            int rl1[kRounds], ro1[kRounds];
+            load_tab(w1, it1, das1, rl1, ro1);
             // ---- finish unit i: clamp, validate, scan, publish ----
-            const int slot = ui & 1;
-            if (ui >= 2) {
-                ok = mbar_wait_warp(&misc->desc_empty[slot], ((ui >> 1) & 1) ^ 1, misc);
+            if (ui >= 1) {                               // the pipeline's consumers have copied the previous descriptor
+                ok = mbar_wait_warp(&misc->desc_empty[x], (ui - 1) & 1, misc);
                 if (!ok) break;
             }
-            UnitDesc& d = misc->desc[slot];
             const bool live = w0 < n_units;
+            int cs[kRounds], len[kRounds], off[kRounds];
             int carry = 0, bad = 0;
 #pragma unroll
             for (int r = 0; r < kRounds; ++r) {
@@ -540,88 +423,169 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     const int v = __shfl_up_sync(0xffffffffu, incl, s);
                     if (lane >= s) incl += v;
                 }
-                d.cs[b] = static_cast<uint16_t>(carry + incl - np4);
+                cs[r] = carry + incl - np4; len[r] = n; off[r] = o;
+                d.cs[b] = static_cast<uint16_t>(cs[r]);
                 d.len[b] = static_cast<uint16_t>(n);
-                d.off[b] = o;
                 carry += __shfl_sync(0xffffffffu, incl, 31);
             }
             if (__any_sync(0xffffffffu, bad) && lane == 0 && p.a.dev_status) atomicOr(p.a.dev_status, HPD_S_BAD_TABLE);
+            Unit u;
+            u.np = live ? (it0.key_count + kN - 1) / kN : 0;
+            u.nt = live ? u.np + (carry + kN - 1) / kN : -1;
+            u.stot = carry; u.head = w0 % Hkv; u.key_count = it0.key_count; u.part_base = it0.part_base;
+            u.row_begin = it0.row_begin; u.nb = it0.row_count;
+            u.row0 = das0 + it0.row_begin; u.kv_row0 = dks0 + it0.key_begin;
             if (lane == 0) {
-                const int np = live ? (it0.key_count + kN - 1) / kN : 0;
-                d.nt = live ? np + (carry + kN - 1) / kN : -1;
-                d.np = np; d.stot = carry;
-                d.head = w0 % Hkv; d.key_count = it0.key_count; d.part_base = it0.part_base;
-                d.row_begin = it0.row_begin; d.nb = it0.row_count;
-                d.row0 = das0 + it0.row_begin; d.kv_row0 = dks0 + it0.key_begin;
+                d.nt = u.nt; d.np = u.np; d.stot = u.stot; d.head = u.head; d.key_count = u.key_count; d.part_base = u.part_base;
+                d.row_begin = u.row_begin; d.nb = u.nb; d.row0 = u.row0; d.kv_row0 = u.kv_row0;
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(&misc->desc_full[slot]);
-            // ---- V tiles of the unit published one iteration ago (its descriptor slot is rewritten only after this) ----
-            if (ui >= 1) {
-                const UnitDesc& dv = misc->desc[slot ^ 1];
-                const Unit uv = read_unit(dv);
-                int vcs[kRounds], vlen[kRounds], voff[kRounds];
-#pragma unroll
-                for (int r = 0; r < kRounds; ++r) { vcs[r] = dv.cs[lane + 32 * r]; vlen[r] = dv.len[lane + 32 * r]; voff[r] = dv.off[lane + 32 * r]; }
-                for (int t = 0; t < uv.nt && ok; ++t) {
-                    const int vs = vc % C::NV;
-                    ok = mbar_wait_warp(&misc->v_empty[vs], ((vc / C::NV) & 1) ^ 1, misc);
-                    if (!ok) break;
-                    fill_tile<D, true>(uv, t, vcs, vlen, voff, lane, smem + C::OFF_V + vs * C::KV_BYTES, &misc->v_full[vs], &map_v, smaps.v);
-                    ++vc;
-                    __syncwarp();
-                }
-            }
+            if (lane == 0) mbar_arrive(&misc->desc_full[x]);
             if (!live) break;
+            // ---- the unit's tiles: K runs one tile ahead of V, the order in which the MMA warp consumes them ----
+            const int nt = u.nt;
+            for (int t = 0; t <= nt && ok; ++t) {
+                if (t < nt) {
+                    const int ks = kc % C::NK;
+                    ok = mbar_wait_warp(&misc->k_empty[x][ks], ((kc / C::NK) & 1) ^ 1, misc);
+                    if (!ok) break;
+                    fill_tile<D, false>(u, t, cs, len, off, lane, k_ring + ks * C::KV_BYTES, &misc->k_full[x][ks], &map_k, smaps.k);
+                    ++kc;
+                    if (t == 0) {
+                        // The Q tile is asked for after the unit's first K tile: its buffer is released late in the
+                        // previous unit, and waiting for it first would hold up the tile that can be fetched already.
+                        ok = mbar_wait_warp(&misc->q_empty[x], (qc & 1) ^ 1, misc);
+                        if (!ok) break;
+                        if (lane == 0) {
+                            mbar_expect_tx(&misc->q_full[x], C::Q_BYTES);
+                            for (int h = 0; h < C::HALVES; ++h)
+                                tma_load_4d(q_tile + h * kQHalf, &map_q, &misc->q_full[x], h * 64, 0, u.head, u.row0);
+                        }
+                        ++qc;
+                    }
+                }
+                if (t >= 1) {
+                    const int vs = vc % C::NV;
+                    ok = mbar_wait_warp(&misc->v_empty[x][vs], ((vc / C::NV) & 1) ^ 1, misc);
+                    if (!ok) break;
+                    fill_tile<D, true>(u, t - 1, cs, len, off, lane, v_ring + vs * C::KV_BYTES, &misc->v_full[x][vs], &map_v, smaps.v);
+                    ++vc;
+                }
+                __syncwarp();
+            }
             // ---- shift the pipeline ----
-            w0 = w1; w1 = w2; w2 = w3; w3 = w4; w4 = w5;
-            it0 = it1; it1 = it2; it2 = it3; it3 = it4;
-            das0 = das1; dks0 = dks1; das1 = das2; dks1 = dks2; das2 = das3; dks2 = dks3;
+            w0 = w1; w1 = w2; w2 = w3; w3 = w4;
+            it0 = it1; it1 = it2; it2 = it3;
+            das0 = das1; dks0 = dks1; das1 = das2; dks1 = dks2;
 #pragma unroll
-            for (int r = 0; r < kRounds; ++r) { rl0[r] = rl1[r]; ro0[r] = ro1[r]; rl1[r] = rl2[r]; ro1[r] = ro2[r]; }
+            for (int r = 0; r < kRounds; ++r) { rl0[r] = rl1[r]; ro0[r] = ro1[r]; }
         }
+        }
+    } else if (warp < 3) {
+        // ================================ MMA issuers (one per pipeline) =============================
+        reg_dealloc<kRegsIo>();
+        if (lane == 0) {
+            const int x = warp - 1;
+            uint32_t qc = 0, tiles = 0;                   // units with tiles so far; tiles of earlier units
+            uint32_t sc = 0, pc = 0;                      // S tiles issued, P tiles consumed
+            bool ok = true;
+            const uint32_t p_lo = desc_lo_kmajor(smem_u32(smem + C::OFF_P + x * kPBytes));
+            const uint32_t q_lo = desc_lo_kmajor(smem_u32(smem + C::OFF_Q + x * C::Q_BYTES));
+            const uint32_t k_lo0 = desc_lo_kmajor(smem_u32(smem + C::OFF_K + x * C::NK * C::KV_BYTES));
+            const uint32_t v_lo0 = desc_lo_mnmajor(smem_u32(smem + C::OFF_V + x * C::NV * C::KV_BYTES));
+            const uint32_t tmem_s = tmem + kColS + x * kN, tmem_o = tmem + kColO + x * 128;
+            const uint32_t idesc_pv = make_idesc(D, 1);
+            for (uint32_t ui = 0; ok; ++ui) {
+                ok = mbar_wait(&misc->desc_full[x], ui & 1, misc);
+                if (!ok) break;
+                const Unit u = read_unit(misc->desc[x]);
+                mbar_arrive(&misc->desc_empty[x]);
+                if (u.nt < 0) break;
+                const int nt = u.nt;
+                if (nt == 0) continue;
+                const int ns = nt - u.np;
+                // columns of tile j: only the last suffix tile and the last prefix tile can be partial
+                const int last_s = u.stot - (ns - 1) * kN, last_p = u.key_count - (u.np - 1) * kN;
+                auto cols16 = [&](int j) { return ((j == ns - 1 ? last_s : (j == nt - 1 ? last_p : kN)) + 15) >> 4; };
+                ok = mbar_wait(&misc->q_full[x], qc & 1, misc);
+                ++qc;
+                auto issue_qk = [&](int j) {
+                    const uint32_t kt = tiles + j;
+                    const int ks = kt % C::NK;
+                    const uint32_t idesc = make_idesc(cols16(j) << 4, 0);
+                    const uint32_t k_lo = k_lo0 + ks * (C::KV_BYTES >> 4);
+                    if (!mbar_wait(&misc->k_full[x][ks], (kt / C::NK) & 1, misc)) return false;
+                    if (!mbar_wait(&misc->s_empty[x], (sc & 1) ^ 1, misc)) return false;
+                    tc_fence_after();
+#pragma unroll
+                    for (int k = 0; k < D / 16; ++k) {
+                        const uint32_t qoff = ((k >> 2) * kQHalf + (k & 3) * 32) >> 4;
+                        const uint32_t koff = ((k >> 2) * kKHalf + (k & 3) * 32) >> 4;
+                        tc_mma(tmem_s, q_lo + qoff, k_lo + koff, idesc, k > 0);
+                    }
+                    tc_commit(&misc->k_empty[x][ks]);
+                    tc_commit(&misc->s_full[x]);
+                    if (j + 1 >= nt) tc_commit(&misc->q_empty[x]);      // last use of the Q tile
+                    ++sc;
+                    return true;
+                };
+                if (ok) ok = issue_qk(0);
+                for (int j = 0; j < nt && ok; ++j) {
+                    if (j + 1 < nt) { ok = issue_qk(j + 1); if (!ok) break; }
+                    const uint32_t vt = tiles + j;
+                    const int vs = vt % C::NV;
+                    const uint32_t v_lo = v_lo0 + vs * (C::KV_BYTES >> 4);
+                    const int nk = cols16(j);
+                    const uint32_t acc0 = j >= 1;
+                    ok = mbar_wait(&misc->p_full[x], pc & 1, misc);
+                    if (!ok) break;
+                    ok = mbar_wait(&misc->v_full[x][vs], (vt / C::NV) & 1, misc);
+                    if (!ok) break;
+                    if (j == 0 && ui > 0) {               // the previous unit's epilogue has read O
+                        ok = mbar_wait(&misc->o_free[x], (ui - 1) & 1, misc);
+                        if (!ok) break;
+                    }
+                    tc_fence_after();
+#pragma unroll
+                    for (int k = 0; k < kN / 16; ++k)
+                        if (k < nk) tc_mma(tmem_o, p_lo + k * 2, v_lo + k * 128, idesc_pv, k > 0 ? 1u : acc0);
+                    tc_commit(&misc->v_empty[x][vs]);
+                    tc_commit(&misc->p_empty[x]);
+                    if (j + 1 >= nt) tc_commit(&misc->o_full[x]);
+                    ++pc;
+                }
+                tiles += nt;
+            }
         }
     } else {
-        // ===================================== softmax A / B ========================================
+        // ======================================= softmax A / B =======================================
         reg_alloc<kRegsSoftmax>();
-        const int x = warp >= 8 ? 1 : 0;                 // stream: even / odd tiles
+        const int x = warp >= 8 ? 1 : 0;                 // pipeline
         const int quad = warp & 3;                       // TMEM lane quadrant this warp may access
         const int row = quad * 32 + lane;                // tile row = TMEM lane
         const uint32_t lane_base = static_cast<uint32_t>(quad * 32) << 16;
         const uint32_t tmem_s = tmem + lane_base + kColS + x * kN;
         const uint32_t tmem_o = tmem + lane_base + kColO + x * 128;
-        // Each stream owns two P tiles and alternates between them, so a new P tile is written while the tensor core
-        // still reads the previous one.  pw counts the P tiles this stream has written so far, pw_other those of the other stream (the groups keep both
-        // counts: the epilogue finds the other stream's (max, sum) area in that stream's next P tile).
-        uint8_t* p_base = smem + C::OFF_P + x * 2 * kPBytes;
+        uint8_t* p_tile = smem + C::OFF_P + x * kPBytes;
         const int b_row = row / G;                       // branch of this row inside the unit
         const uint32_t g_magic = 0xFFFFFFFFu / static_cast<uint32_t>(G) + 1u;   // floor(r / G) = umulhi(r, g_magic) for r < 2^16, G > 1
-        uint32_t s_cnt = 0;
-        uint32_t pw = 0, pw_other = 0;
-        uint32_t of_a = 0, of_b = 0;
+        uint32_t s_cnt = 0, pw = 0, of_cnt = 0;          // S tiles read, P tiles written, units with tiles
         bool ok = true;
         for (uint32_t unit_idx = 0; ok; ++unit_idx) {
-            const int slot = unit_idx & 1;
-            ok = mbar_wait_warp(&misc->desc_full[slot], (unit_idx >> 1) & 1, misc);
+            ok = mbar_wait_warp(&misc->desc_full[x], unit_idx & 1, misc);
             if (!ok) break;
-            const Unit u = read_unit(misc->desc[slot]);
+            const Unit u = read_unit(misc->desc[x]);
             // packed columns [my_cs, my_cs + my_len) hold this row's own cached tokens
-            const int my_cs = misc->desc[slot].cs[b_row], my_len = misc->desc[slot].len[b_row];
+            const int my_cs = misc->desc[x].cs[b_row], my_len = misc->desc[x].len[b_row];
             __syncwarp();
-            if (lane == 0) mbar_arrive(&misc->desc_empty[slot]);
+            if (lane == 0) mbar_arrive(&misc->desc_empty[x]);
             if (u.nt < 0) break;
             const int nt = u.nt;
             const int nrows = u.nb * G;
             const bool row_valid = row < nrows;
             const bool warp_active = quad * 32 < nrows;
-            const int n_mine = (nt + 1 - x) >> 1;
-            if (unit_idx > 0) {                          // P buffers and O are free again
-                ok = mbar_wait_warp(&misc->o_free, (unit_idx - 1) & 1, misc);
-                if (!ok) break;
-            }
             float m = -INFINITY, l = 0.f;
-            for (int i = 0; i < n_mine && ok; ++i) {
-                const int j = x + 2 * i;
+            for (int j = 0; j < nt && ok; ++j) {
                 // Columns of this tile the row may see.  A suffix tile holds a few branches each; a warp whose rows see
                 // none of them (known from the descriptor alone) skips the tile's scores and writes zero probabilities.
                 int lo = 0, hi = 0;
@@ -650,6 +614,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&misc->s_empty[x]);
 
+                bool waited = false;
                 if (vis) {
                     if (!__all_sync(0xffffffffu, lo == 0 && hi == kN)) {
                         const unsigned span = static_cast<unsigned>(hi - lo);
@@ -666,15 +631,16 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         for (int k = 0; k < 8; ++k) t8[k] = fmax3(t8[k], __uint_as_float(sv[c + k]), __uint_as_float(sv[c + 8 + k]));
                     float tmax = fmax3(fmax3(t8[0], t8[1], t8[2]), fmax3(t8[3], t8[4], t8[5]), fmaxf(t8[6], t8[7]));
                     tmax *= p.scale_log2;
-                    if (i == 0) {
+                    if (j == 0) {
                         m = tmax;
                     } else {
                         const bool fresh = m == -INFINITY;       // nothing visible so far: O row is still exactly zero
                         if (fresh) m = tmax;
                         const bool grow = !fresh && tmax > m + kRescaleSlack;
                         if (__any_sync(0xffffffffu, grow)) {
-                            // O must be rescaled: wait until this stream's previous P V product has landed in TMEM
-                            ok = mbar_wait_warp(&misc->p_empty[x * 2 + ((pw - 1) & 1)], ((pw - 1) >> 1) & 1, misc);
+                            // O must be rescaled: wait until the previous P V product has landed in TMEM
+                            ok = mbar_wait_warp(&misc->p_empty[x], (pw - 1) & 1, misc);
+                            waited = true;
                             if (ok) {
                                 tc_fence_after();
                                 const float m_new = grow ? tmax : m;
@@ -695,18 +661,18 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         }
                     }
                 }
-                const int pb = pw & 1;                 // the P V product that read this P tile two tiles ago is done
-                ok = ok && mbar_wait_warp(&misc->p_empty[x * 2 + pb], ((pw >> 1) & 1) ^ 1, misc);
+                if (pw > 0 && !waited)                   // the previous P V product has consumed the P tile
+                    ok = ok && mbar_wait_warp(&misc->p_empty[x], (pw - 1) & 1, misc);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 if (warp_active && !vis) {              // nothing visible for any row of the warp: P rows of zeros
-                    uint8_t* prow = p_base + pb * kPBytes + row * 128;
+                    uint8_t* prow = p_tile + row * 128;
 #pragma unroll
                     for (int kc8 = 0; kc8 < kN / 8; ++kc8) *reinterpret_cast<uint4*>(prow + (kc8 << 4)) = make_uint4(0, 0, 0, 0);
                     fence_async_smem();
                 } else if (warp_active) {
                     const float neg_m = (m == -INFINITY) ? 0.f : -m;
-                    uint8_t* prow = p_base + pb * kPBytes + row * 128;
+                    uint8_t* prow = p_tile + row * 128;
                     float lsum[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                     for (int kc8 = 0; kc8 < kN / 8; ++kc8) {
@@ -726,78 +692,47 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&misc->p_full[x * 2 + pb]);
+                if (lane == 0) mbar_arrive(&misc->p_full[x]);
                 ++pw;
             }
             if (!ok) break;
 
             // ------------------------------------ epilogue ------------------------------------
-            // both groups merge the two streams; group x writes output columns [x*D/2, (x+1)*D/2)
-            pw_other += (nt + x) >> 1;                 // tiles the other stream writes in this unit
-            // the stream's next P tile is idle until the next unit: it carries the (max, sum) exchange and the output staging
-            ok = mbar_wait_warp(&misc->p_empty[x * 2 + (pw & 1)], ((pw >> 1) & 1) ^ 1, misc);
-            if (!ok) break;
-            uint8_t* p_tile = p_base + (pw & 1) * kPBytes;
-            float2* ml_mine = reinterpret_cast<float2*>(p_tile);
-            const float2* ml_other = reinterpret_cast<const float2*>(smem + C::OFF_P + ((x ^ 1) * 2 + (pw_other & 1)) * kPBytes);
-            const float2* ml_a = x == 0 ? ml_mine : ml_other;
-            const float2* ml_b = x == 0 ? ml_other : ml_mine;
-            ml_mine[row] = make_float2(m, l);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&misc->ml_full);
-            ok = mbar_wait_warp(&misc->ml_full, unit_idx & 1, misc);
-            if (!ok) break;
-            const int n_a = (nt + 1) >> 1, n_b = nt >> 1;
-            if (n_a > 0) { ok = mbar_wait_warp(&misc->o_full[0], of_a & 1, misc); ++of_a; if (!ok) break; }
-            if (n_b > 0) { ok = mbar_wait_warp(&misc->o_full[1], of_b & 1, misc); ++of_b; if (!ok) break; }
+            if (nt > 0) {                                // the unit's last P V product has landed (and the P tile is free)
+                ok = mbar_wait_warp(&misc->o_full[x], of_cnt & 1, misc);
+                ++of_cnt;
+                if (!ok) break;
+            }
             tc_fence_after();
-
-            const float2 sa = ml_a[row], sb = ml_b[row];
-            const float mt = fmaxf(sa.x, sb.x);
-            const float fa = sa.x == -INFINITY ? 0.f : ex2(sa.x - mt);
-            const float fb = sb.x == -INFINITY ? 0.f : ex2(sb.x - mt);
-            const float lt = fa * sa.y + fb * sb.y;
-
-            constexpr int HC = D / 2;                    // columns of this group's half
             const int g_row = row - b_row * G;
             const int grow_row = u.row0 + b_row;
             const int hq = u.head * G + g_row;
             const bool store = row_valid && grow_row < p.a.max_rows;
             const bool final_out = u.part_base < 0;
-            const float inv = final_out ? (lt > 0.f ? 1.f / lt : 0.f) : 1.f;
-            const float ca = fa * inv, cb = fb * inv;
+            const float inv = final_out ? (l > 0.f ? 1.f / l : 0.f) : 1.f;
             const int64_t pr = (static_cast<int64_t>(final_out ? 0 : u.part_base) + u.row_begin + b_row) * p.a.g.Hq + hq;
-            float* po = p.part_o + pr * D + x * HC;
+            float* po = p.part_o + pr * D;
 #pragma unroll
-            for (int c0 = 0; c0 < HC; c0 += 32) {
+            for (int c0 = 0; c0 < D; c0 += 32) {
                 float acc[32];
 #pragma unroll
                 for (int c = 0; c < 32; ++c) acc[c] = 0.f;
-                if (warp_active) {
-                    if (n_a > 0 && n_b > 0) {            // both streams: the two loads are in flight together
-                        uint32_t oa[32], ob[32];
-                        tmem_ld32(tmem + lane_base + kColO + x * HC + c0, oa);
-                        tmem_ld32(tmem + lane_base + kColO + 128 + x * HC + c0, ob);
-                        tmem_ld_wait();
+                if (warp_active && nt > 0) {
+                    uint32_t ov[32];
+                    tmem_ld32(tmem_o + c0, ov);
+                    tmem_ld_wait();
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) acc[c] = fmaf(cb, __uint_as_float(ob[c]), ca * __uint_as_float(oa[c]));
-                    } else if (n_a > 0) {
-                        uint32_t ov[32];
-                        tmem_ld32(tmem + lane_base + kColO + x * HC + c0, ov);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) acc[c] = ca * __uint_as_float(ov[c]);
-                    }
+                    for (int c = 0; c < 32; ++c) acc[c] = inv * __uint_as_float(ov[c]);
                 }
-                if (c0 + 32 >= HC) {                     // all TMEM reads of this unit are done
+                if (c0 + 32 >= D) {                      // all TMEM reads of this unit are done
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&misc->o_free);
+                    if (lane == 0) mbar_arrive(&misc->o_free[x]);
                 }
                 if (final_out) {
-                    // transpose through shared memory (2 KB inside this warp's own rows of the stream's idle P tile,
-                    // past the (max, sum) exchange area): a row's 32 columns go out as one 64-byte piece, 8 rows per store
-                    uint8_t* stg = p_tile + quad * 4096 + 1024;
+                    // transpose through shared memory (2 KB inside this warp's own rows of the idle P tile): a row's
+                    // 32 columns go out as one 64-byte piece, 8 rows per store instruction
+                    uint8_t* stg = p_tile + quad * 4096;
 #pragma unroll
                     for (int c = 0; c < 32; c += 8) {
                         uint4 pk;
@@ -816,7 +751,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         const int tb = G == 1 ? trow : static_cast<int>(__umulhi(static_cast<uint32_t>(trow), g_magic)), tg = trow - tb * G;
                         const int grow = u.row0 + tb;
                         if (trow < nrows && grow < p.a.max_rows)
-                            *reinterpret_cast<uint4*>(p.a.o + (static_cast<int64_t>(grow) * p.a.g.Hq + u.head * G + tg) * D + x * HC + c0 + ch * 8) = pk;
+                            *reinterpret_cast<uint4*>(p.a.o + (static_cast<int64_t>(grow) * p.a.g.Hq + u.head * G + tg) * D + c0 + ch * 8) = pk;
                     }
                     __syncwarp();
                 } else if (store) {
@@ -825,11 +760,11 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         *reinterpret_cast<float4*>(po + c0 + c) = make_float4(acc[c], acc[c + 1], acc[c + 2], acc[c + 3]);
                 }
             }
-            if (store && x == 0) {
+            if (store) {
                 if (final_out) {
-                    if (p.a.lse) p.a.lse[static_cast<int64_t>(grow_row) * p.a.g.Hq + hq] = lt > 0.f ? (mt + log2f(lt)) * kLn2 : -INFINITY;
+                    if (p.a.lse) p.a.lse[static_cast<int64_t>(grow_row) * p.a.g.Hq + hq] = l > 0.f ? (m + log2f(l)) * kLn2 : -INFINITY;
                 } else {
-                    p.part_ml[pr * 2] = mt; p.part_ml[pr * 2 + 1] = lt;
+                    p.part_ml[pr * 2] = m; p.part_ml[pr * 2 + 1] = l;
                 }
             }
         }
