@@ -45,7 +45,9 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleSlack = 8.0f;      // tolerated growth of the row maximum (log2 units) before O is rescaled
 constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz
-constexpr uint32_t kColS = 0, kColO = 128;
+// TMEM columns of one pipeline (the second pipeline's start 256 columns further): scores, two probability tiles
+// (bf16 pairs, 32 columns each), output accumulator
+constexpr uint32_t kColPipe = 256, kColS = 0, kColP = 64, kColO = 128;
 // registers per thread after the warpgroups have traded them (3 x 128 threads, 168 each at launch)
 constexpr int kRegsIo = 96, kRegsSoftmax = 200;
 // setmaxnreg only moves registers inside the CTA's own allocation (168 x 384 threads at launch): a request beyond
@@ -64,8 +66,8 @@ template <int D> struct Cfg {
     static constexpr int NK = D == 128 ? 2 : 4;                  // K stages of each pipeline
     static constexpr int NV = D == 128 ? 2 : 4;                  // V stages of each pipeline
     static constexpr int OFF_Q = 0;                              // one Q tile per pipeline
-    static constexpr int OFF_P = OFF_Q + 2 * Q_BYTES;           // one P tile per pipeline
-    static constexpr int OFF_K = OFF_P + 2 * kPBytes;
+    static constexpr int OFF_STAGE = OFF_Q + 2 * Q_BYTES;       // output transpose, 2 KB per softmax warp
+    static constexpr int OFF_K = OFF_STAGE + 8 * 2048;
     static constexpr int OFF_V = OFF_K + 2 * NK * KV_BYTES;
     static constexpr int OFF_MISC = OFF_V + 2 * NV * KV_BYTES;
     static constexpr int SMEM = OFF_MISC + 3072;                 // + misc; the dynamic segment itself is 1024-B aligned
@@ -111,7 +113,7 @@ static_assert(sizeof(UnitDesc) == 48 + 4 * kM, "descriptor size");
 struct Misc {
     unsigned long long q_full[2], q_empty[2];
     unsigned long long k_full[2][kMaxStages], k_empty[2][kMaxStages], v_full[2][kMaxStages], v_empty[2][kMaxStages];
-    unsigned long long s_full[2], s_empty[2], p_full[2], p_empty[2], o_full[2], o_free[2];
+    unsigned long long s_full[2], s_empty[2], p_full[2][2], p_empty[2][2], o_full[2], o_free[2];
     unsigned long long desc_full[2], desc_empty[2];
     uint32_t tmem_base;
     int abort_flag;
@@ -186,6 +188,14 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint32_t a_lo, uint32_t 
                  "mov.b64 da, {%1, %5};\n\tmov.b64 db, {%2, %5};\n\tsetp.ne.b32 p, %4, 0;\n\t"
                  "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
                  ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(0x40004040u) : "memory");
+}
+
+// The same with the A operand in tensor memory (the probabilities, written there by the softmax threads).
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+                 "mov.b64 db, {%2, %5};\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(0x40004040u) : "memory");
 }
 
 #define HPD_R8(a, o) "=r"(a[o + 0]), "=r"(a[o + 1]), "=r"(a[o + 2]), "=r"(a[o + 3]), "=r"(a[o + 4]), "=r"(a[o + 5]), "=r"(a[o + 6]), "=r"(a[o + 7])
@@ -313,7 +323,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         for (int i = 0; i < 2; ++i) {
             mbar_init(&misc->q_full[i], 1);  mbar_init(&misc->q_empty[i], 1);
             mbar_init(&misc->s_full[i], 1);  mbar_init(&misc->s_empty[i], 4);
-            mbar_init(&misc->p_full[i], 4);  mbar_init(&misc->p_empty[i], 1);
+            for (int b = 0; b < 2; ++b) { mbar_init(&misc->p_full[i][b], 4); mbar_init(&misc->p_empty[i][b], 1); }
             mbar_init(&misc->o_full[i], 1);  mbar_init(&misc->o_free[i], 4);
             mbar_init(&misc->desc_full[i], 1); mbar_init(&misc->desc_empty[i], kDescReaders);
             for (int k = 0; k < kMaxStages; ++k) {
@@ -489,11 +499,10 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             uint32_t qc = 0, tiles = 0;                   // units with tiles so far; tiles of earlier units
             uint32_t sc = 0, pc = 0;                      // S tiles issued, P tiles consumed
             bool ok = true;
-            const uint32_t p_lo = desc_lo_kmajor(smem_u32(smem + C::OFF_P + x * kPBytes));
             const uint32_t q_lo = desc_lo_kmajor(smem_u32(smem + C::OFF_Q + x * C::Q_BYTES));
             const uint32_t k_lo0 = desc_lo_kmajor(smem_u32(smem + C::OFF_K + x * C::NK * C::KV_BYTES));
             const uint32_t v_lo0 = desc_lo_mnmajor(smem_u32(smem + C::OFF_V + x * C::NV * C::KV_BYTES));
-            const uint32_t tmem_s = tmem + kColS + x * kN, tmem_o = tmem + kColO + x * 128;
+            const uint32_t tmem_s = tmem + x * kColPipe + kColS, tmem_p = tmem + x * kColPipe + kColP, tmem_o = tmem + x * kColPipe + kColO;
             const uint32_t idesc_pv = make_idesc(D, 1);
             for (uint32_t ui = 0; ok; ++ui) {
                 ok = mbar_wait(&misc->desc_full[x], ui & 1, misc);
@@ -537,7 +546,8 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     const uint32_t v_lo = v_lo0 + vs * (C::KV_BYTES >> 4);
                     const int nk = cols16(j);
                     const uint32_t acc0 = j >= 1;
-                    ok = mbar_wait(&misc->p_full[x], pc & 1, misc);
+                    const int pb = pc & 1;
+                    ok = mbar_wait(&misc->p_full[x][pb], (pc >> 1) & 1, misc);
                     if (!ok) break;
                     ok = mbar_wait(&misc->v_full[x][vs], (vt / C::NV) & 1, misc);
                     if (!ok) break;
@@ -548,9 +558,9 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     tc_fence_after();
 #pragma unroll
                     for (int k = 0; k < kN / 16; ++k)
-                        if (k < nk) tc_mma(tmem_o, p_lo + k * 2, v_lo + k * 128, idesc_pv, k > 0 ? 1u : acc0);
+                        if (k < nk) tc_mma_ts(tmem_o, tmem_p + pb * 32 + k * 8, v_lo + k * 128, idesc_pv, k > 0 ? 1u : acc0);
                     tc_commit(&misc->v_empty[x][vs]);
-                    tc_commit(&misc->p_empty[x]);
+                    tc_commit(&misc->p_empty[x][pb]);
                     if (j + 1 >= nt) tc_commit(&misc->o_full[x]);
                     ++pc;
                 }
@@ -564,9 +574,10 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const int quad = warp & 3;                       // TMEM lane quadrant this warp may access
         const int row = quad * 32 + lane;                // tile row = TMEM lane
         const uint32_t lane_base = static_cast<uint32_t>(quad * 32) << 16;
-        const uint32_t tmem_s = tmem + lane_base + kColS + x * kN;
-        const uint32_t tmem_o = tmem + lane_base + kColO + x * 128;
-        uint8_t* p_tile = smem + C::OFF_P + x * kPBytes;
+        const uint32_t tmem_s = tmem + lane_base + x * kColPipe + kColS;
+        const uint32_t tmem_p = tmem + lane_base + x * kColPipe + kColP;
+        const uint32_t tmem_o = tmem + lane_base + x * kColPipe + kColO;
+        uint8_t* stg = smem + C::OFF_STAGE + (x * 4 + quad) * 2048;      // this warp's output staging
         const int b_row = row / G;                       // branch of this row inside the unit
         const uint32_t g_magic = 0xFFFFFFFFu / static_cast<uint32_t>(G) + 1u;   // floor(r / G) = umulhi(r, g_magic) for r < 2^16, G > 1
         uint32_t s_cnt = 0, pw = 0, of_cnt = 0;          // S tiles read, P tiles written, units with tiles
@@ -614,7 +625,6 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&misc->s_empty[x]);
 
-                bool waited = false;
                 if (vis) {
                     if (!__all_sync(0xffffffffu, lo == 0 && hi == kN)) {
                         const unsigned span = static_cast<unsigned>(hi - lo);
@@ -639,8 +649,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         const bool grow = !fresh && tmax > m + kRescaleSlack;
                         if (__any_sync(0xffffffffu, grow)) {
                             // O must be rescaled: wait until the previous P V product has landed in TMEM
-                            ok = mbar_wait_warp(&misc->p_empty[x], (pw - 1) & 1, misc);
-                            waited = true;
+                            ok = mbar_wait_warp(&misc->p_empty[x][(pw - 1) & 1], ((pw - 1) >> 1) & 1, misc);
                             if (ok) {
                                 tc_fence_after();
                                 const float m_new = grow ? tmax : m;
@@ -661,38 +670,35 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         }
                     }
                 }
-                if (pw > 0 && !waited)                   // the previous P V product has consumed the P tile
-                    ok = ok && mbar_wait_warp(&misc->p_empty[x], (pw - 1) & 1, misc);
+                const int pb = pw & 1;                   // the P V product that read this P tile two tiles ago is done
+                ok = ok && mbar_wait_warp(&misc->p_empty[x][pb], ((pw >> 1) & 1) ^ 1, misc);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                if (warp_active && !vis) {              // nothing visible for any row of the warp: P rows of zeros
-                    uint8_t* prow = p_tile + row * 128;
+                // Probabilities go to tensor memory as bf16 pairs (column c of the P tile holds keys 2c and 2c+1 of the
+                // row), from where the tensor core reads them as the A operand of O += P V.
+                if (warp_active) {
+                    uint32_t pk[kN / 2];
+                    if (!vis) {                          // nothing visible for any row of the warp: zero probabilities
 #pragma unroll
-                    for (int kc8 = 0; kc8 < kN / 8; ++kc8) *reinterpret_cast<uint4*>(prow + (kc8 << 4)) = make_uint4(0, 0, 0, 0);
-                    fence_async_smem();
-                } else if (warp_active) {
-                    const float neg_m = (m == -INFINITY) ? 0.f : -m;
-                    uint8_t* prow = p_tile + row * 128;
-                    float lsum[4] = {0.f, 0.f, 0.f, 0.f};
+                        for (int c = 0; c < kN / 2; ++c) pk[c] = 0u;
+                    } else {
+                        const float neg_m = (m == -INFINITY) ? 0.f : -m;
+                        float lsum[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                    for (int kc8 = 0; kc8 < kN / 8; ++kc8) {
-                        float e[8];
-#pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            e[q] = ex2(fmaf(__uint_as_float(sv[kc8 * 8 + q]), p.scale_log2, neg_m));
-                            lsum[q & 3] += e[q];
+                        for (int c = 0; c < kN / 2; ++c) {
+                            const float e0 = ex2(fmaf(__uint_as_float(sv[2 * c]), p.scale_log2, neg_m));
+                            const float e1 = ex2(fmaf(__uint_as_float(sv[2 * c + 1]), p.scale_log2, neg_m));
+                            lsum[c & 1] += e0; lsum[2 + (c & 1)] += e1;
+                            pk[c] = pack_bf16(e0, e1);
                         }
-                        uint4 pk;
-                        pk.x = pack_bf16(e[0], e[1]); pk.y = pack_bf16(e[2], e[3]);
-                        pk.z = pack_bf16(e[4], e[5]); pk.w = pack_bf16(e[6], e[7]);
-                        *reinterpret_cast<uint4*>(prow + ((kc8 ^ (row & 7)) << 4)) = pk;
+                        l += (lsum[0] + lsum[1]) + (lsum[2] + lsum[3]);
                     }
-                    l += (lsum[0] + lsum[1]) + (lsum[2] + lsum[3]);
-                    fence_async_smem();
+                    tmem_st32(tmem_p + pb * 32, pk);
+                    tmem_st_wait();
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&misc->p_full[x]);
+                if (lane == 0) mbar_arrive(&misc->p_full[x][pb]);
                 ++pw;
             }
             if (!ok) break;
@@ -730,9 +736,8 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     if (lane == 0) mbar_arrive(&misc->o_free[x]);
                 }
                 if (final_out) {
-                    // transpose through shared memory (2 KB inside this warp's own rows of the idle P tile): a row's
-                    // 32 columns go out as one 64-byte piece, 8 rows per store instruction
-                    uint8_t* stg = p_tile + quad * 4096;
+                    // transpose through this warp's 2 KB of shared memory: a row's 32 columns go out as one 64-byte
+                    // piece, 8 rows per store instruction
 #pragma unroll
                     for (int c = 0; c < 32; c += 8) {
                         uint4 pk;
