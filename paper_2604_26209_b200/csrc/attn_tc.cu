@@ -1,25 +1,29 @@
 // hpd_attn_decode on the 5th-generation tensor cores (tcgen05 + TMEM), fed by TMA.
 //
-// One persistent CTA per SM walks the step's work units.  A unit = (work item, kv head): up to
-// 128/G branches of one document (rows = branches x G query heads, the M dimension) against a chunk
-// of that document's prefix, so each prefix K/V byte is read from HBM once for all of the document's
-// branches.  Keys are consumed in tiles of 64: first the tiles into which the branches' own cached
-// tokens ("suffix") are packed back to back, each branch padded to a multiple of four columns so
-// that one TMA box of 4..16 cache rows places it (the few K rows read beyond a branch's length are
-// masked; V boxes have the exact height), masked block-diagonally (a row sees only its own branch's
-// columns); then the prefix tiles.  The suffix tiles come first because their many small copies are
-// slow to issue and can be issued while the previous unit is still in its epilogue.  Even tiles form
-// stream A, odd tiles stream B, each with its own MMA-issuing warp, softmax group, score buffer,
-// pair of probability tiles and output accumulator, so the two streams run as independent
-// online-softmax pipelines over one K/V stream (a split-KV inside the CTA); the epilogue merges them.
+// One persistent CTA per SM runs two independent pipelines, each of which walks work units of its
+// own.  A unit = (work item, kv head): up to 128/G branches of one document (rows = branches x G
+// query heads, the M dimension) against a chunk of that document's prefix, so each prefix K/V byte
+// is read from HBM once for all of the document's branches.  Keys are consumed in tiles of 64:
+// first the tiles into which the branches' own cached tokens ("suffix") are packed back to back,
+// each branch padded to a multiple of four columns so that one TMA box of 4..16 cache rows places
+// it (the few K rows read beyond a branch's length are masked; V boxes have the exact height),
+// masked block-diagonally (a row sees only its own branch's columns); then the prefix tiles.  The
+// suffix tiles come first because their many small copies are slow to issue and can be issued
+// while the pipeline's previous unit is still being finished.
 //
-//   warp 0        TMA producer of the Q tile and the K tiles (prefix: lane 0; suffix boxes: all lanes)
-//   warps 1-2     MMA issuers of streams A and B: S = Q K^T and O += P V (tcgen05.mma, TMEM accumulators)
-//   warp 3        scheduler (draws units, publishes their descriptors) and TMA producer of the V tiles
-//   warps 4-7     softmax A     one thread per row: S from TMEM, online max/sum, P (bf16) to shared
-//   warps 8-11    softmax B     memory, rare rescale of O in TMEM; both groups share the epilogue
+// Per unit a pipeline is latency-bound (one thread per row in the softmax, one thread issuing the
+// MMAs, a serial epilogue); two of them on one SM overlap each other's waits and epilogues, which
+// is what keeps HBM busy.  A pipeline owns a Q tile, a K and a V ring (shared memory), a score
+// tile, two probability tiles and an output accumulator (tensor memory), and these warps:
 //
-// TMEM columns: S_A [0,64)  S_B [64,128)  O_A [128,256)  O_B [256,384).
+//   warp 0 / 3    scheduler and TMA producer: draws the pipeline's units, publishes their
+//                 descriptors, issues Q, K and V tiles (prefix: lane 0; suffix boxes: all lanes)
+//   warp 1 / 2    MMA issuer: S = Q K^T (both operands in shared memory) and O += P V (P in tensor
+//                 memory, V in shared memory); tcgen05.mma, accumulators in tensor memory
+//   warps 4-7 /   softmax: one thread per row: S from TMEM, online max/sum, P (bf16 pairs) to TMEM,
+//   warps 8-11    rare rescale of O in TMEM; epilogue: O / sum -> bf16 -> shared -> global
+//
+// TMEM columns of a pipeline (second pipeline + 256): S [0,64)  P0 [64,96)  P1 [96,128)  O [128,256).
 //
 // All waits are bounded: a wait that gives up raises HPD_S_TIMEOUT in the status word and the CTA
 // drains and exits (TMEM is released on every path).
@@ -40,7 +44,6 @@ constexpr int kM = 128;                    // rows of a tile
 constexpr int kN = 64;                     // keys of a tile
 constexpr int kQHalf = kM * 128;           // one 64-element half of the Q tile: 128 rows x 128 B
 constexpr int kKHalf = kN * 128;           // one 64-element half of a K or V tile: 64 keys x 128 B
-constexpr int kPBytes = kM * 128;          // P tile: 128 rows x 64 keys bf16
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleSlack = 8.0f;      // tolerated growth of the row maximum (log2 units) before O is rescaled
@@ -91,11 +94,11 @@ struct TcParams {
 };
 
 // ------------------------------------------------------------------------------------------------
-// Unit descriptors.  One warp (the scheduler) draws work units from the step's ticket counter, gathers
+// Unit descriptors.  A pipeline's producer warp draws work units from the step's ticket counter, gathers
 // everything the other roles need to know about a unit -- tile counts, first rows, and per branch the
-// number of cached tokens, the first cache row and the packed column of its first token -- and publishes
-// it in one of two shared-memory slots.  Every other warp copies what it needs into registers at the start
-// of the unit and releases the slot at once, so no role ever waits for a dependent global load.
+// number of cached tokens and the packed column of its first token -- and publishes it in the pipeline's
+// shared-memory slot.  The MMA thread and the softmax warps copy what they need into registers at the start
+// of the unit and release the slot at once, so no role ever waits for a dependent global load.
 // ------------------------------------------------------------------------------------------------
 struct UnitDesc {
     int nt;          // tiles of the unit (prefix + suffix); -1: no more units
@@ -210,6 +213,10 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* v) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
                  "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
                  ::"r"(taddr), HPD_W8(v, 0), HPD_W8(v, 8), HPD_W8(v, 16), HPD_W8(v, 24) : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* v) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+                 ::"r"(taddr), HPD_W8(v, 0), HPD_W8(v, 8) : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
@@ -677,23 +684,29 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 // Probabilities go to tensor memory as bf16 pairs (column c of the P tile holds keys 2c and 2c+1 of the
                 // row), from where the tensor core reads them as the A operand of O += P V.
                 if (warp_active) {
-                    uint32_t pk[kN / 2];
                     if (!vis) {                          // nothing visible for any row of the warp: zero probabilities
+                        uint32_t pk[16];
 #pragma unroll
-                        for (int c = 0; c < kN / 2; ++c) pk[c] = 0u;
+                        for (int c = 0; c < 16; ++c) pk[c] = 0u;
+                        tmem_st16(tmem_p + pb * 32, pk);
+                        tmem_st16(tmem_p + pb * 32 + 16, pk);
                     } else {
                         const float neg_m = (m == -INFINITY) ? 0.f : -m;
                         float lsum[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                        for (int c = 0; c < kN / 2; ++c) {
-                            const float e0 = ex2(fmaf(__uint_as_float(sv[2 * c]), p.scale_log2, neg_m));
-                            const float e1 = ex2(fmaf(__uint_as_float(sv[2 * c + 1]), p.scale_log2, neg_m));
-                            lsum[c & 1] += e0; lsum[2 + (c & 1)] += e1;
-                            pk[c] = pack_bf16(e0, e1);
+                        for (int h = 0; h < 2; ++h) {    // 32 keys = 16 columns of bf16 pairs per store
+                            uint32_t pk[16];
+#pragma unroll
+                            for (int c = 0; c < 16; ++c) {
+                                const float e0 = ex2(fmaf(__uint_as_float(sv[h * 32 + 2 * c]), p.scale_log2, neg_m));
+                                const float e1 = ex2(fmaf(__uint_as_float(sv[h * 32 + 2 * c + 1]), p.scale_log2, neg_m));
+                                lsum[c & 1] += e0; lsum[2 + (c & 1)] += e1;
+                                pk[c] = pack_bf16(e0, e1);
+                            }
+                            tmem_st16(tmem_p + pb * 32 + h * 16, pk);
                         }
                         l += (lsum[0] + lsum[1]) + (lsum[2] + lsum[3]);
                     }
-                    tmem_st32(tmem_p + pb * 32, pk);
                     tmem_st_wait();
                 }
                 tc_fence_before();
