@@ -48,9 +48,9 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleSlack = 8.0f;      // tolerated growth of the row maximum (log2 units) before O is rescaled
 constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz
-// TMEM columns of one pipeline (the second pipeline's start 256 columns further): scores, two probability tiles
-// (bf16 pairs, 32 columns each), output accumulator
-constexpr uint32_t kColPipe = 256, kColS = 0, kColP = 64, kColO = 128;
+// TMEM columns of one pipeline (the second pipeline's start 256 columns further): two score tiles of 64 columns (the
+// probabilities of a tile, bf16 pairs, overwrite the first 32 columns of its scores) and the output accumulator
+constexpr uint32_t kColPipe = 256, kColS = 0, kColO = 128;
 // registers per thread after the warpgroups have traded them (3 x 128 threads, 168 each at launch)
 constexpr int kRegsIo = 96, kRegsSoftmax = 200;
 // setmaxnreg only moves registers inside the CTA's own allocation (168 x 384 threads at launch): a request beyond
@@ -116,7 +116,7 @@ static_assert(sizeof(UnitDesc) == 48 + 4 * kM, "descriptor size");
 struct Misc {
     unsigned long long q_full[2], q_empty[2];
     unsigned long long k_full[2][kMaxStages], k_empty[2][kMaxStages], v_full[2][kMaxStages], v_empty[2][kMaxStages];
-    unsigned long long s_full[2], s_empty[2], p_full[2][2], p_empty[2][2], o_full[2], o_free[2];
+    unsigned long long s_full[2][2], p_full[2][2], p_empty[2][2], o_full[2], o_free[2];
     unsigned long long desc_full[2], desc_empty[2];
     uint32_t tmem_base;
     int abort_flag;
@@ -329,8 +329,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     if (threadIdx.x == 0) {
         for (int i = 0; i < 2; ++i) {
             mbar_init(&misc->q_full[i], 1);  mbar_init(&misc->q_empty[i], 1);
-            mbar_init(&misc->s_full[i], 1);  mbar_init(&misc->s_empty[i], 4);
-            for (int b = 0; b < 2; ++b) { mbar_init(&misc->p_full[i][b], 4); mbar_init(&misc->p_empty[i][b], 1); }
+            for (int b = 0; b < 2; ++b) { mbar_init(&misc->s_full[i][b], 1); mbar_init(&misc->p_full[i][b], 4); mbar_init(&misc->p_empty[i][b], 1); }
             mbar_init(&misc->o_full[i], 1);  mbar_init(&misc->o_free[i], 4);
             mbar_init(&misc->desc_full[i], 1); mbar_init(&misc->desc_empty[i], kDescReaders);
             for (int k = 0; k < kMaxStages; ++k) {
@@ -509,7 +508,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             const uint32_t q_lo = desc_lo_kmajor(smem_u32(smem + C::OFF_Q + x * C::Q_BYTES));
             const uint32_t k_lo0 = desc_lo_kmajor(smem_u32(smem + C::OFF_K + x * C::NK * C::KV_BYTES));
             const uint32_t v_lo0 = desc_lo_mnmajor(smem_u32(smem + C::OFF_V + x * C::NV * C::KV_BYTES));
-            const uint32_t tmem_s = tmem + x * kColPipe + kColS, tmem_p = tmem + x * kColPipe + kColP, tmem_o = tmem + x * kColPipe + kColO;
+            const uint32_t tmem_s = tmem + x * kColPipe + kColS, tmem_o = tmem + x * kColPipe + kColO;
             const uint32_t idesc_pv = make_idesc(D, 1);
             for (uint32_t ui = 0; ok; ++ui) {
                 ok = mbar_wait(&misc->desc_full[x], ui & 1, misc);
@@ -531,23 +530,24 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     const uint32_t idesc = make_idesc(cols16(j) << 4, 0);
                     const uint32_t k_lo = k_lo0 + ks * (C::KV_BYTES >> 4);
                     if (!mbar_wait(&misc->k_full[x][ks], (kt / C::NK) & 1, misc)) return false;
-                    if (!mbar_wait(&misc->s_empty[x], (sc & 1) ^ 1, misc)) return false;
                     tc_fence_after();
 #pragma unroll
                     for (int k = 0; k < D / 16; ++k) {
                         const uint32_t qoff = ((k >> 2) * kQHalf + (k & 3) * 32) >> 4;
                         const uint32_t koff = ((k >> 2) * kKHalf + (k & 3) * 32) >> 4;
-                        tc_mma(tmem_s, q_lo + qoff, k_lo + koff, idesc, k > 0);
+                        tc_mma(tmem_s + (sc & 1) * kN, q_lo + qoff, k_lo + koff, idesc, k > 0);
                     }
                     tc_commit(&misc->k_empty[x][ks]);
-                    tc_commit(&misc->s_full[x]);
+                    tc_commit(&misc->s_full[x][sc & 1]);
                     if (j + 1 >= nt) tc_commit(&misc->q_empty[x]);      // last use of the Q tile
                     ++sc;
                     return true;
                 };
+                // Scores run two tiles ahead: S(j+2) overwrites the tile in which S(j) was computed and P(j) was read,
+                // and the tensor core executes this thread's MMAs in the order of issue, P(j) V(j) before it.
                 if (ok) ok = issue_qk(0);
+                if (ok && nt > 1) ok = issue_qk(1);
                 for (int j = 0; j < nt && ok; ++j) {
-                    if (j + 1 < nt) { ok = issue_qk(j + 1); if (!ok) break; }
                     const uint32_t vt = tiles + j;
                     const int vs = vt % C::NV;
                     const uint32_t v_lo = v_lo0 + vs * (C::KV_BYTES >> 4);
@@ -565,11 +565,12 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     tc_fence_after();
 #pragma unroll
                     for (int k = 0; k < kN / 16; ++k)
-                        if (k < nk) tc_mma_ts(tmem_o, tmem_p + pb * 32 + k * 8, v_lo + k * 128, idesc_pv, k > 0 ? 1u : acc0);
+                        if (k < nk) tc_mma_ts(tmem_o, tmem_s + pb * kN + k * 8, v_lo + k * 128, idesc_pv, k > 0 ? 1u : acc0);
                     tc_commit(&misc->v_empty[x][vs]);
                     tc_commit(&misc->p_empty[x][pb]);
                     if (j + 1 >= nt) tc_commit(&misc->o_full[x]);
                     ++pc;
+                    if (j + 2 < nt) ok = issue_qk(j + 2);
                 }
                 tiles += nt;
             }
@@ -581,13 +582,12 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const int quad = warp & 3;                       // TMEM lane quadrant this warp may access
         const int row = quad * 32 + lane;                // tile row = TMEM lane
         const uint32_t lane_base = static_cast<uint32_t>(quad * 32) << 16;
-        const uint32_t tmem_s = tmem + lane_base + x * kColPipe + kColS;
-        const uint32_t tmem_p = tmem + lane_base + x * kColPipe + kColP;
+        const uint32_t tmem_s0 = tmem + lane_base + x * kColPipe + kColS;
         const uint32_t tmem_o = tmem + lane_base + x * kColPipe + kColO;
         uint8_t* stg = smem + C::OFF_STAGE + (x * 4 + quad) * 2048;      // this warp's output staging
         const int b_row = row / G;                       // branch of this row inside the unit
         const uint32_t g_magic = 0xFFFFFFFFu / static_cast<uint32_t>(G) + 1u;   // floor(r / G) = umulhi(r, g_magic) for r < 2^16, G > 1
-        uint32_t s_cnt = 0, pw = 0, of_cnt = 0;          // S tiles read, P tiles written, units with tiles
+        uint32_t pw = 0, of_cnt = 0;                     // tiles done (S read, P written), units with tiles
         bool ok = true;
         for (uint32_t unit_idx = 0; ok; ++unit_idx) {
             ok = mbar_wait_warp(&misc->desc_full[x], unit_idx & 1, misc);
@@ -619,18 +619,16 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     }
                 }
                 const bool vis = __any_sync(0xffffffffu, hi > lo);
-                ok = mbar_wait_warp(&misc->s_full[x], s_cnt & 1, misc);
+                const int pb = pw & 1;                   // the tile's S / P buffer
+                const uint32_t tmem_s = tmem_s0 + pb * kN;
+                ok = mbar_wait_warp(&misc->s_full[x][pb], (pw >> 1) & 1, misc);
                 if (!ok) break;
-                ++s_cnt;
                 tc_fence_after();
                 uint32_t sv[kN];
                 if (vis) {
                     tmem_ld32(tmem_s, sv); tmem_ld32(tmem_s + 32, sv + 32);
                     tmem_ld_wait();
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&misc->s_empty[x]);
 
                 if (vis) {
                     if (!__all_sync(0xffffffffu, lo == 0 && hi == kN)) {
@@ -677,19 +675,17 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         }
                     }
                 }
-                const int pb = pw & 1;                   // the P V product that read this P tile two tiles ago is done
-                ok = ok && mbar_wait_warp(&misc->p_empty[x][pb], ((pw >> 1) & 1) ^ 1, misc);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                // Probabilities go to tensor memory as bf16 pairs (column c of the P tile holds keys 2c and 2c+1 of the
-                // row), from where the tensor core reads them as the A operand of O += P V.
+                // Probabilities go to tensor memory as bf16 pairs (column c holds keys 2c and 2c+1 of the row), over the
+                // first half of the row's own scores, from where the tensor core reads them as the A operand of O += P V.
                 if (warp_active) {
                     if (!vis) {                          // nothing visible for any row of the warp: zero probabilities
                         uint32_t pk[16];
 #pragma unroll
                         for (int c = 0; c < 16; ++c) pk[c] = 0u;
-                        tmem_st16(tmem_p + pb * 32, pk);
-                        tmem_st16(tmem_p + pb * 32 + 16, pk);
+                        tmem_st16(tmem_s, pk);
+                        tmem_st16(tmem_s + 16, pk);
                     } else {
                         const float neg_m = (m == -INFINITY) ? 0.f : -m;
                         float lsum[4] = {0.f, 0.f, 0.f, 0.f};
@@ -703,7 +699,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                                 lsum[c & 1] += e0; lsum[2 + (c & 1)] += e1;
                                 pk[c] = pack_bf16(e0, e1);
                             }
-                            tmem_st16(tmem_p + pb * 32 + h * 16, pk);
+                            tmem_st16(tmem_s + h * 16, pk);
                         }
                         l += (lsum[0] + lsum[1]) + (lsum[2] + lsum[3]);
                     }
