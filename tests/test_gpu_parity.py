@@ -130,6 +130,22 @@ def test_step_matches_oracle(rt, name):
     assert np.max(np.abs(lse_gpu - want.lse)) <= 2e-2
 
 
+def test_attention_is_bitwise_reproducible_across_launches(rt):
+    """Work units are handed to the kernel's two pipelines per SM by a ticket counter, so which pipeline computes a
+    row changes from launch to launch; the tiles of a unit are always taken in the same order, so the bits must not."""
+    s = synth.config_main(n_prompts=8)                  # more units than pipelines: the ticket counter is in use
+    tb = synth.make_tensors(s)
+    db, tabs = _run_step(rt, s, tb)
+    n = tabs["n_active"]
+    o0, l0 = rt.bits_of(db.o)[:n].copy(), db.lse.cpu().numpy()[:n].copy()
+    for _ in range(3):
+        db.attn(True)
+        torch.cuda.synchronize()
+        assert db.status() == 0
+        assert np.array_equal(rt.bits_of(db.o)[:n], o0)
+        assert np.array_equal(db.lse.cpu().numpy()[:n], l0)
+
+
 @pytest.mark.parametrize("name", ["tiny", "main_p2", "ragged", "ragged_d64_g2", "long_small"])
 def test_std_decode_matches_oracle_and_hpd(rt, name):
     s = STRUCTS[name]()
