@@ -43,6 +43,10 @@ STRUCTS = {
     "one_group_96": lambda: synth.config_custom("wide", Hq=32, Hkv=8, D=128, theta=500000.0, cap=8,
                                                 prefix_lens=[700], branch_cnts=[96], depth_hi=8, seed=6),
     "few_alive": lambda: _ragged(7, alive_frac=0.1),
+    # more documents than the single-launch table builder takes: the three-kernel path
+    "many_docs": lambda: synth.config_custom("many", Hq=2, Hkv=1, D=64, theta=10000.0, cap=4,
+                                             prefix_lens=[(7 * i) % 23 for i in range(4300)],
+                                             branch_cnts=[(i % 3) for i in range(4300)], depth_hi=4, seed=10, alive_frac=0.7),
     # one query head per kv head: 128 branches per unit, four rounds of branch tables, dozens of suffix tiles per unit
     "g1_many_branches": lambda: synth.config_custom("g1", Hq=2, Hkv=2, D=128, theta=10000.0, cap=32,
                                                     prefix_lens=[200, 50, 0], branch_cnts=[200, 130, 70], depth_hi=32, seed=9),
