@@ -377,13 +377,15 @@ def run_loop(args):
     n_act = [int((s.eos_len > t).sum()) for t in range(steps)]
     stream = torch.cuda.current_stream()
 
+    t_dev = torch.zeros((), dtype=torch.int32, device=dev)      # step counter on the device (the graph advances it)
+
     def one_step(t):
-        # caller-side state of the loop (which branches are still decoding, how deep they are)
-        torch.minimum(eos, torch.full_like(eos, t), out=depth)
-        alive.copy_((eos > t).to(torch.uint8))
+        # caller-side state of the loop (which branches are still decoding, how deep they are); t: host int or t_dev
+        torch.minimum(eos, t_dev if t is None else torch.full_like(eos, t), out=depth)
+        alive.copy_((eos > (t_dev if t is None else t)).to(torch.uint8))
         B.hpd_build_meta(g, s.n_docs, s.n_slots, L_d, cnt, depth, alive, 0, meta)
         for l in range(L):
-            b = (t + l) & 1
+            b = l & 1
             B.hpd_rope(g, s.n_slots, meta.n_active, meta.pos_id, q[b], kn[b])
             B.hpd_kv_append(g, s.n_slots, s.n_slots, meta.n_active, meta.suffix_off, meta.suffix_len, kn[b], vn[b],
                             suf_k[l], suf_v[l], meta.dev_status)
@@ -394,10 +396,22 @@ def run_loop(args):
         one_step(t)
     torch.cuda.synchronize()
     sampler = ClockSampler(0); sampler.start(); time.sleep(0.3)
+    graph = None
+    if not args.no_graph:
+        # one decode step (table build + all layers) captured once; the step counter lives on the device
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            one_step(None)
+            t_dev.add_(1)
+        t_dev.zero_()
+        torch.cuda.synchronize()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
     ev[0].record(stream)
     for t in range(steps):
-        one_step(t)
+        if graph is not None:
+            graph.replay()
+        else:
+            one_step(t)
         ev[t + 1].record(stream)
     torch.cuda.synchronize()
     clocks = sampler.stop()
@@ -409,7 +423,8 @@ def run_loop(args):
         "ms_per_step": total_ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic", "config": {"workload": f"{s.name}_L{L}", "layers": L, "prompts": s.n_prompts,
                                         "branches_per_prompt": 96, "suffix_cap": g.suffix_cap,
-                                        "l2": "inputs larger than L2 (every layer has its own caches); no flush"},
+                                        "l2": "inputs larger than L2 (every layer has its own caches); no flush",
+                                        "launch": "cuda graph replay of one decode step" if graph is not None else "direct calls"},
         "clocks": clocks, "gpu_launches": steps * (3 + 4 * L), "dev_status": int(meta.dev_status.item()),
         "per_layer_branch_tokens_per_s": tokens * L / (total_ms * 1e-3),
         "series": [{"step": t, "n_active": n_act[t], "ms": ms[t]} for t in range(steps)],
