@@ -214,10 +214,8 @@ def run_ours(args):
     # ---- the same step replayed from a CUDA graph (extra information: launch-bound small batches) ---------
     ms_graph = None
     if not args.no_graph:
-        g = torch.cuda.CUDAGraph()
         barrier()
-        with torch.cuda.graph(g):
-            db.step(with_meta=True)
+        g = db.capture_step(with_meta=True)
         for _ in range(3):
             g.replay()
         barrier()

@@ -80,6 +80,15 @@ class DeviceBatch:
         self.kv_append()
         self.attn(True)
 
+    def capture_step(self, with_meta=True):
+        """The step's launches captured once in a CUDA graph (call step() at least once before: the first call sets
+        kernel attributes and builds tensor maps).  replay() then runs the same kernels without a host call each."""
+        g = torch.cuda.CUDAGraph()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g):
+            self.step(with_meta=with_meta)
+        return g
+
     # -- read-back --------------------------------------------------------------------------
     def tables(self) -> Dict[str, np.ndarray]:
         s = self.s

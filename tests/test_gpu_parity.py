@@ -134,6 +134,24 @@ def test_step_matches_oracle(rt, name):
     assert np.max(np.abs(lse_gpu - want.lse)) <= 2e-2
 
 
+def test_graph_replay_equals_direct_calls(rt):
+    """The step captured in a CUDA graph launches the same kernels on the same buffers: same bits."""
+    s = synth.config_main(n_prompts=2)
+    tb = synth.make_tensors(s)
+    db, tabs = _run_step(rt, s, tb)
+    n = tabs["n_active"]
+    act = tabs["active_slot"][:n]
+    o0 = rt.bits_of(db.o)[:n].copy()
+    g = db.capture_step(with_meta=True)
+    for _ in range(2):
+        db.set_step_inputs(tb["q"][act], tb["k_new"][act], tb["v_new"][act])     # rope rotates q and k in place
+        db.o.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert db.status() == 0
+        assert np.array_equal(rt.bits_of(db.o)[:n], o0)
+
+
 def test_attention_is_bitwise_reproducible_across_launches(rt):
     """Work units are handed to the kernel's two pipelines per SM by a ticket counter, so which pipeline computes a
     row changes from launch to launch; the tiles of a unit are always taken in the same order, so the bits must not."""
