@@ -52,9 +52,9 @@ constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz
 // probabilities of a tile, bf16 pairs, overwrite the first 32 columns of its scores) and the output accumulator
 constexpr uint32_t kColPipe = 256, kColS = 0, kColO = 128;
 // registers per thread after the warpgroups have traded them (3 x 128 threads, 168 each at launch)
-constexpr int kRegsIo = 96, kRegsSoftmax = 200;
+constexpr int kRegsIo = 104, kRegsSoftmax = 200;
 // setmaxnreg only moves registers inside the CTA's own allocation (168 x 384 threads at launch): a request beyond
-// that pool would block forever
+// that pool would block forever; using the pool exactly is fine
 static_assert(kRegsIo + 2 * kRegsSoftmax <= 3 * 168, "registers traded between the warpgroups exceed the CTA's allocation");
 constexpr int kBoxKinds = 4;               // suffix boxes of 4, 8, 12, 16 cache rows
 constexpr int kPad = 4;                    // a branch's cached tokens occupy a multiple of 4 packed columns
