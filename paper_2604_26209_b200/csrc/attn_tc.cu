@@ -373,9 +373,9 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             if (lane == 0) { d.nt = -1; mbar_arrive(&misc->desc_full[x]); }
         } else {
         // The first units of a pipeline are fixed (unit = 2 * CTA + pipeline + i * 2 * grid), which fills the software
-        // pipeline without a chain of atomics; later units are drawn from the step's ticket counter, so faster SMs
-        // (and the pipeline that got shorter units) take more.
-        constexpr int kStatic = 5;
+        // pipeline without a chain of atomics and measured slightly faster than drawing early; later units are drawn
+        // from the step's ticket counter, so faster SMs (and the pipeline that got shorter units) take more.
+        constexpr int kStatic = 6;
         const uint32_t first_dynamic = static_cast<uint32_t>(kStatic) * 2u * gridDim.x;
         auto draw = [&]() {                              // next unit index (lane 0 draws, all lanes get it)
             uint32_t t = 0;
@@ -409,7 +409,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         bool ok = true;
         for (uint32_t ui = 0; ok; ++ui) {
             // ---- issue the next stage of every unit in flight (results are used in the next iteration) ----
-            const int w4 = ui == 0 ? fixed(4) : draw();
+            const int w4 = static_cast<int>(ui) + 4 < kStatic ? fixed(static_cast<int>(ui) + 4) : draw();
             const WorkItem it3 = item_of(w3);
             const int das2 = p.a.doc_active_start[it2.doc], dks2 = p.a.doc_kv_start[it2.doc];
             int rl1[kRounds], ro1[kRounds];
