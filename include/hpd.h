@@ -34,7 +34,8 @@ extern "C" {
 #endif
 
 /* Attention geometry.  Supported: D in {64, 128}; Hq % Hkv == 0 with G in {1, 2, 4, 8};
- * 1 <= suffix_cap.  sm_scale multiplies q.k before the softmax (1/sqrt(D) in the paper's
+ * 1 <= suffix_cap, and for hpd_attn_decode (128/G) * round_up(suffix_cap, 4) <= 65535 (i.e. suffix_cap
+ * <= 508 / 1020 / 2044 / 4092 for G = 1 / 2 / 4 / 8; larger slabs return HPD_E_CAPACITY).  sm_scale multiplies q.k before the softmax (1/sqrt(D) in the paper's
  * "scaled dot-product attention", Sec. 4.3.2).  suffix_cap is the branch-cache slab size in
  * tokens: the K_max of Sec. 4.3.1 (values longer than K_max are truncated, Sec. 4.3.4). */
 typedef struct hpd_geom {
@@ -48,7 +49,7 @@ enum {
     HPD_E_ARG       = -1,   /* null / misaligned pointer, negative size                        */
     HPD_E_GEOM      = -2,   /* geometry outside the supported set                              */
     HPD_E_WORKSPACE = -3,   /* workspace_bytes smaller than hpd_workspace_bytes() reports      */
-    HPD_E_CAPACITY  = -4,   /* a size exceeds what the call can index (int32 tables)           */
+    HPD_E_CAPACITY  = -4,   /* a size exceeds what the call can index (int32 tables, slab size) */
     HPD_E_CUDA      = -5    /* a CUDA runtime/driver call failed; see hpd_last_cuda_error()    */
 };
 
@@ -174,7 +175,12 @@ int std_attn_decode(const hpd_geom* geom /*host*/, int max_rows, int max_seq_len
  *     nothing is launched; use std_attn_decode with your own workspace then.
  *   - The call allocates nothing (no cudaMalloc/cudaFree, no allocating library routine).
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) and keeps
- *     it; make that first call outside any stream capture.
+ *     it; make that first call outside any stream capture.  It is also the moment at which the CUDA
+ *     runtime may place the library's device image, the array included, on that device, which can fail
+ *     when the device heap is already exhausted: make one warm-up call at start-up, before memory gets
+ *     tight.  From then on a call takes nothing from the device heap.
+ *   - One process may use the library on several devices; every per-device cache of the library (this
+ *     address, SM counts, kernel attributes) is keyed by the device that is current at the call.
  *   - All calls on one device share the array and it keeps the last call's contents.  Nothing needs
  *     clearing (each call writes every partial before its merge reads it), but two calls whose
  *     kernels can overlap on the GPU (different streams) race on it: keep them on one stream or

@@ -1,6 +1,5 @@
 // extern "C" entry points of libhpd (see include/hpd.h): argument checks and kernel dispatch only.
-#include <cstdlib>
-#include <cstring>
+#include <atomic>
 
 #include "common.cuh"
 
@@ -21,29 +20,31 @@ int geom_check(const hpd_geom* g)
     return HPD_OK;
 }
 
+int current_device()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+    return dev;
+}
+
+// SM count of the current device.  Looked up once per device; the table is only ever written with the value the
+// driver reports for that device, so concurrent first calls store the same number.
 int sm_count()
 {
-    static int cached = 0;
-    if (cached > 0) return cached;
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) {
-        cached = n;
+    static std::atomic<int> cached[kMaxDevices];
+    const int dev = current_device();
+    const bool slot = dev >= 0 && dev < kMaxDevices;
+    if (slot) {
+        const int c = cached[dev].load(std::memory_order_relaxed);
+        if (c > 0) return c;
+    }
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) {
+        if (slot) cached[dev].store(n, std::memory_order_relaxed);
         return n;
     }
     (void)cudaGetLastError();
     return 148;
-}
-
-// HPD_ATTN_IMPL=simt forces the scalar kernel in hpd_attn_decode (debugging aid).
-static bool force_simt()
-{
-    static int v = -1;
-    if (v < 0) {
-        const char* e = std::getenv("HPD_ATTN_IMPL");
-        v = (e && std::strcmp(e, "simt") == 0) ? 1 : 0;
-    }
-    return v == 1;
 }
 
 }  // namespace hpd
@@ -59,7 +60,7 @@ const char* hpd_strerror(int code)
         case HPD_E_ARG: return "invalid argument (null or misaligned pointer, negative size)";
         case HPD_E_GEOM: return "unsupported geometry (need D in {64,128}, Hq/Hkv in {1,2,4,8}, suffix_cap >= 1)";
         case HPD_E_WORKSPACE: return "workspace too small";
-        case HPD_E_CAPACITY: return "size exceeds int32 table range";
+        case HPD_E_CAPACITY: return "size exceeds what the call can index (int32 tables; suffix_cap too large for the attention kernel)";
         case HPD_E_CUDA: return "CUDA call failed (see hpd_last_cuda_error)";
         default: return "unknown error code";
     }
@@ -140,6 +141,8 @@ int hpd_attn_decode(const hpd_geom* geom, int n_docs, int max_rows, int n_slots,
 {
     int rc = geom_check(geom);
     if (rc != HPD_OK) return rc;
+    // the attention kernel keeps each branch's packed column and cached-token count as 16-bit numbers
+    if (attn_packed_columns(*geom) > kMaxPackedColumns) return HPD_E_CAPACITY;
     if (n_docs < 0 || max_rows < 0 || n_slots < 0 || total_prefix_tokens < 0) return HPD_E_ARG;
     if (max_rows == 0 || n_docs == 0) return HPD_OK;
     if (!q || !suffix_k || !suffix_v || !doc_kv_start || !doc_prefix_len || !doc_active_start || !doc_id ||
@@ -150,35 +153,22 @@ int hpd_attn_decode(const hpd_geom* geom, int n_docs, int max_rows, int n_slots,
     const WsLayout lay = ws_layout(*geom, n_docs, n_slots, sm_count());
     if (workspace_bytes < lay.total) return HPD_E_WORKSPACE;
 
-    if (!force_simt()) {
-        AttnArgs a{};
-        a.g = *geom;
-        a.n_docs = n_docs; a.max_rows = max_rows; a.n_slots = n_slots; a.total_prefix = total_prefix_tokens;
-        a.q = static_cast<const __nv_bfloat16*>(q);
-        a.prefix_k = static_cast<const __nv_bfloat16*>(prefix_k);
-        a.prefix_v = static_cast<const __nv_bfloat16*>(prefix_v);
-        a.suffix_k = static_cast<const __nv_bfloat16*>(suffix_k);
-        a.suffix_v = static_cast<const __nv_bfloat16*>(suffix_v);
-        a.doc_kv_start = doc_kv_start; a.doc_prefix_len = doc_prefix_len; a.doc_active_start = doc_active_start;
-        a.doc_id = doc_id; a.suffix_off = suffix_off; a.suffix_len = suffix_len; a.n_active = n_active;
-        a.suffix_extra = suffix_includes_new ? 1 : 0;
-        a.o = static_cast<__nv_bfloat16*>(o);
-        a.lse = lse;
-        a.workspace = workspace; a.lay = lay; a.dev_status = dev_status;
-        a.stream = static_cast<cudaStream_t>(stream);
-        return launch_attn_tc(a);
-    }
-    SimtArgs s{};
-    s.g = *geom;
-    s.max_rows = max_rows; s.n_splits = 1; s.n_active = n_active;
-    s.q = static_cast<const __nv_bfloat16*>(q);
-    s.k1 = static_cast<const __nv_bfloat16*>(prefix_k); s.v1 = static_cast<const __nv_bfloat16*>(prefix_v);
-    s.doc_id = doc_id; s.doc_kv_start = doc_kv_start; s.doc_prefix_len = doc_prefix_len;
-    s.k2 = static_cast<const __nv_bfloat16*>(suffix_k); s.v2 = static_cast<const __nv_bfloat16*>(suffix_v);
-    s.suffix_off = suffix_off; s.suffix_len = suffix_len; s.suffix_extra = suffix_includes_new ? 1 : 0;
-    s.o = static_cast<__nv_bfloat16*>(o); s.lse = lse; s.part = nullptr;
-    s.stream = static_cast<cudaStream_t>(stream);
-    return launch_attn_simt(s);
+    AttnArgs a{};
+    a.g = *geom;
+    a.n_docs = n_docs; a.max_rows = max_rows; a.n_slots = n_slots; a.total_prefix = total_prefix_tokens;
+    a.q = static_cast<const __nv_bfloat16*>(q);
+    a.prefix_k = static_cast<const __nv_bfloat16*>(prefix_k);
+    a.prefix_v = static_cast<const __nv_bfloat16*>(prefix_v);
+    a.suffix_k = static_cast<const __nv_bfloat16*>(suffix_k);
+    a.suffix_v = static_cast<const __nv_bfloat16*>(suffix_v);
+    a.doc_kv_start = doc_kv_start; a.doc_prefix_len = doc_prefix_len; a.doc_active_start = doc_active_start;
+    a.doc_id = doc_id; a.suffix_off = suffix_off; a.suffix_len = suffix_len; a.n_active = n_active;
+    a.suffix_extra = suffix_includes_new ? 1 : 0;
+    a.o = static_cast<__nv_bfloat16*>(o);
+    a.lse = lse;
+    a.workspace = workspace; a.lay = lay; a.dev_status = dev_status;
+    a.stream = static_cast<cudaStream_t>(stream);
+    return launch_attn_tc(a);
 }
 
 static int std_splits(const hpd_geom* g, int max_rows, int max_seq_len)

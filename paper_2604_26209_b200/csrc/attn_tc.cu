@@ -13,23 +13,26 @@
 //
 // Per unit a pipeline is latency-bound (one thread per row in the softmax, one thread issuing the
 // MMAs, a serial epilogue); two of them on one SM overlap each other's waits and epilogues, which
-// is what keeps HBM busy.  A pipeline owns a Q tile, a K and a V ring (shared memory), a score
-// tile, two probability tiles and an output accumulator (tensor memory), and these warps:
+// is what keeps HBM busy.  A pipeline owns a Q tile, a K and a V ring (shared memory), two score
+// tiles and an output accumulator (tensor memory), and these warps:
 //
 //   warp 0 / 3    scheduler and TMA producer: draws the pipeline's units, publishes their
 //                 descriptors, issues Q, K and V tiles (prefix: lane 0; suffix boxes: all lanes)
-//   warp 1 / 2    MMA issuer: S = Q K^T (both operands in shared memory) and O += P V (P in tensor
-//                 memory, V in shared memory); tcgen05.mma, accumulators in tensor memory
-//   warps 4-7 /   softmax: one thread per row: S from TMEM, online max/sum, P (bf16 pairs) to TMEM,
-//   warps 8-11    rare rescale of O in TMEM; epilogue: O / sum -> bf16 -> shared -> global
+//   warp 1 / 2    MMA issuer: S = Q K^T (both operands in shared memory), two tiles ahead of the
+//                 softmax, and O += P V (P in tensor memory, V in shared memory); tcgen05.mma
+//   warps 4-7 /   softmax: one thread per row: S from TMEM, online max/sum, P as bf16 pairs written
+//   warps 8-11    over the first half of the row's own scores, rare rescale of O in TMEM; epilogue:
+//                 O / sum -> bf16 -> shared -> global
 //
-// TMEM columns of a pipeline (second pipeline + 256): S [0,64)  P0 [64,96)  P1 [96,128)  O [128,256).
+// TMEM columns of a pipeline (second pipeline + 256): S0 [0,64)  S1 [64,128)  O [128,256); the
+// probabilities of a tile occupy the first 32 columns of the score tile they were computed from.
 //
 // All waits are bounded: a wait that gives up raises HPD_S_TIMEOUT in the status word and the CTA
 // drains and exits (TMEM is released on every path).
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "common.cuh"
@@ -901,10 +904,12 @@ template <int D>
 int launch_d(const AttnArgs& a)
 {
     using C = Cfg<D>;
-    static bool attr_set = false;
-    if (!attr_set) {
+    // the dynamic shared-memory limit is an attribute of the kernel on ONE device: set it once per device
+    static std::atomic<bool> attr_set[kMaxDevices];
+    const int dev = current_device();
+    if (dev < 0 || dev >= kMaxDevices || !attr_set[dev].load(std::memory_order_acquire)) {
         HPD_CUDA_TRY(cudaFuncSetAttribute(hpd_attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
-        attr_set = true;
+        if (dev >= 0 && dev < kMaxDevices) attr_set[dev].store(true, std::memory_order_release);
     }
     const int G = a.g.Hq / a.g.Hkv;
     // Tensor maps depend only on the tensors' addresses and extents: a decode loop calls with the same ones step

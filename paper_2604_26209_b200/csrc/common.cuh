@@ -25,8 +25,20 @@ void set_last_cuda_error(cudaError_t e);
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+constexpr int kMaxDevices = 64;      // per-device caches (SM count, kernel attributes) are indexed by device ordinal
+
 int geom_check(const hpd_geom* g);   // HPD_OK or HPD_E_GEOM / HPD_E_ARG
+int current_device();                // ordinal of the calling thread's current device (0 if it cannot be queried)
 int sm_count();                      // SMs of the current device (148 if it cannot be queried)
+
+// hpd_attn_decode packs the cached tokens of the up to 128/G branches of a unit back to back, each branch rounded
+// up to a multiple of four columns, and stores a branch's first column and length as 16-bit numbers.
+constexpr long long kMaxPackedColumns = 65535;
+inline long long attn_packed_columns(const hpd_geom& g)
+{
+    const long long G = g.Hq / g.Hkv;
+    return (128 / G) * ((static_cast<long long>(g.suffix_cap) + 3) & ~3ll);
+}
 
 // ---------------------------------------------------------------------------------------------
 // Workspace of one decode step.  hpd_build_meta writes the header and the work list;

@@ -38,6 +38,19 @@ def test_argument_checks_need_no_device():
     assert lib.hpd_workspace_bytes(C.byref(good), 256, 6144, 131072) > 0
 
 
+def test_attention_rejects_slabs_beyond_its_16_bit_column_index():
+    """hpd_attn_decode packs up to 128/G branches of round4(suffix_cap) columns each and indexes them with 16 bits:
+    larger slabs are refused before anything is launched (no pointer is looked at)."""
+    lib = binding.load()
+    nulls = [None] * 12
+    tail = [1, None, None, None, 0, None, None]
+    for Hq, Hkv, cap, want in ((8, 1, 4092, -1), (8, 1, 4093, -4), (32, 8, 2044, -1), (32, 8, 2045, -4),
+                               (4, 4, 508, -1), (4, 4, 512, -4)):
+        g = binding.HpdGeom(Hq, Hkv, 128, 10000.0, 0.1, cap)
+        assert lib.hpd_attn_decode(C.byref(g), 1, 1, 1, 1, *nulls, *tail) == want, (Hq, Hkv, cap)
+    assert b"suffix_cap" in lib.hpd_strerror(-4)
+
+
 def test_missing_library_is_an_error(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "_lib", None)
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))

@@ -1,11 +1,16 @@
-"""Full-size parity on sampled rows: the benchmark workloads in the launch configuration bench.py
-times, checked against the oracle on a sample of rows the oracle computes one by one."""
+"""Full-size parity: the benchmark workloads in the launch configuration bench.py times.
+
+The two workloads the metric is quoted on (64 prompts of the main shape, 32 prompts of the long-document
+shape) are compared with the oracle on EVERY row, with a bound on each row's own error, so that a fault
+confined to a few work units of a fully occupied GPU cannot hide in a sample or in a mean.  The largest
+point of the prompt-batch sweep (256 prompts) is compared on a sample of rows.
+"""
 import numpy as np
 import pytest
 import torch
 
 from paper_2604_26209_b200 import synth
-from tests.util import oracle_step, err_stats
+from tests.util import oracle_step
 
 pytestmark = pytest.mark.gpu
 MAX_ABS, MEAN_ABS = 2e-2, 2e-3
@@ -19,17 +24,7 @@ def rt():
     return runtime
 
 
-@pytest.mark.parametrize("make,n_sample", [(lambda: synth.config_main(n_prompts=64), 96),
-                                           (lambda: synth.config_long(n_prompts=32), 48)])
-def test_fullsize_sampled_rows(rt, make, n_sample):
-    s = make()
-    tb = synth.make_tensors(s)
-    rng = np.random.default_rng(123)
-    rows = np.sort(rng.choice(s.n_active, size=n_sample, replace=False))
-    # make sure first/last rows of documents and of the batch are in the sample
-    rows[:4] = [0, 1, s.n_active - 2, s.n_active - 1]
-    rows = np.unique(rows)
-    meta, want = oracle_step(s, tb, rows=rows)
+def _gpu_step(rt, s, tb):
     db = rt.DeviceBatch(s, tb)
     db.build_meta()
     tabs = db.tables()
@@ -41,10 +36,44 @@ def test_fullsize_sampled_rows(rt, make, n_sample):
     db.attn(True)
     torch.cuda.synchronize()
     assert db.status() == 0
-    o = synth.bf16_bits_to_f32(rt.bits_of(db.o))
-    mx, mean = err_stats(o[rows], want.o)
-    assert mx <= MAX_ABS and mean <= MEAN_ABS, (mx, mean)
-    # properties that hold at any size: every written row is finite; rows beyond n_active untouched
-    assert np.isfinite(o[: s.n_active]).all()
+    o = synth.bf16_bits_to_f32(rt.bits_of(db.o))[: s.n_active]
     lse = db.lse.cpu().numpy()[: s.n_active]
+    return db, tabs, o, lse
+
+
+def _check(o, lse, want, rows):
+    d = np.abs(o[rows].astype(np.float64) - want.o)
+    assert d.max() <= MAX_ABS and d.mean() <= MEAN_ABS, (d.max(), d.mean())
+    per_row_max = d.reshape(len(rows), -1).max(axis=1)
+    per_row_mean = d.reshape(len(rows), -1).mean(axis=1)
+    worst = int(np.argmax(per_row_mean))
+    # a row's own mean error: 3x the bar on the global mean still separates rounding (a few 1e-4) from a wrong key
+    assert per_row_max.max() <= MAX_ABS and per_row_mean.max() <= 3 * MEAN_ABS, (rows[worst], per_row_mean[worst])
     assert np.max(np.abs(lse[rows] - want.lse)) <= 2e-2
+
+
+@pytest.mark.parametrize("make", [lambda: synth.config_main(n_prompts=64), lambda: synth.config_long(n_prompts=32)],
+                         ids=["main_p64", "long_p32"])
+def test_fullsize_every_row(rt, make):
+    s = make()
+    tb = synth.make_tensors(s)
+    meta, want = oracle_step(s, tb)
+    db, tabs, o, lse = _gpu_step(rt, s, tb)
+    from oracle import capi
+    for nm in capi.Meta.TABLES:
+        assert np.array_equal(tabs[nm], getattr(meta, nm)), nm
+    assert np.isfinite(o).all()
+    _check(o, lse, want, np.arange(s.n_active))
+
+
+def test_sweep_largest_batch_sampled_rows(rt):
+    """256 prompts (24576 rows, 8192 work units): rows sampled across the whole batch, first and last rows included."""
+    s = synth.config_main(n_prompts=256)
+    tb = synth.make_tensors(s)
+    rng = np.random.default_rng(321)
+    rows = np.unique(np.concatenate([rng.choice(s.n_active, size=384, replace=False),
+                                     [0, 1, 23, 24, s.n_active - 25, s.n_active - 24, s.n_active - 1]]))
+    meta, want = oracle_step(s, tb, rows=rows)
+    db, tabs, o, lse = _gpu_step(rt, s, tb)
+    assert np.isfinite(o).all()
+    _check(o, lse, want, rows)

@@ -63,3 +63,92 @@ def test_loop_with_ragged_retirement_matches_oracle():
         assert np.all(np.abs(gk[lo:lo + n] - cache_k[lo:lo + n]) <= np.abs(cache_k[lo:lo + n]) * 2.0 ** -8 + 1e-6)
         assert np.array_equal(gv[lo:lo + n], cache_v[lo:lo + n])
         assert np.isnan(gk[lo + n: lo + g.suffix_cap]).all()                # rows beyond the value's length were never written
+
+
+def test_fullsize_loop_two_layers_sampled_branches():
+    """The loop workload at its real batch (64 prompts x 96 branches, cap 32, end-of-value lengths min(Geom(1/8), 32))
+    over ALL steps and two layers with their own caches: tables bit-exact at every step, outputs of a fixed sample of
+    branches against the oracle at every step and layer, final cache contents of those branches.  Under the
+    branch-local mask of Eq. 5-6 a branch's history is its own, so the oracle keeps caches for the sampled branches only."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from dataclasses import replace
+    from paper_2604_26209_b200 import runtime, binding as B
+    L = 2
+    s0 = synth.config_loop(n_prompts=64, seed=5)
+    g, dev = s0.geom, "cuda"
+    cap, kvw = g.suffix_cap, g.Hkv * g.D
+    rng = np.random.default_rng(99)
+    # sample: some long-lived branches (so late steps with few live rows per document are checked), some random ones
+    order = np.argsort(-s0.eos_len, kind="stable")
+    sample = np.unique(np.concatenate([order[:24], rng.choice(s0.n_slots, 72, replace=False), [0, s0.n_slots - 1]]))
+    pools = {k: synth.randn_bf16(rng, (s0.n_slots, h, g.D)) for k, h in (("q", g.Hq), ("k", g.Hkv), ("v", g.Hkv))}
+    pre = [synth.make_tensors(s0, suffix=False, step=False, salt=l) for l in range(L)]
+    f_pre = [{k: synth.bf16_bits_to_f32(v) for k, v in p.items()} for p in pre]
+    bf = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(dev).view(torch.bfloat16)
+    pre_k = [bf(p["prefix_k"]) for p in pre]; pre_v = [bf(p["prefix_v"]) for p in pre]
+    nan = lambda: torch.full((s0.n_slots * cap, g.Hkv, g.D), float("nan"), dtype=torch.bfloat16, device=dev)
+    suf_k = [nan() for _ in range(L)]; suf_v = [nan() for _ in range(L)]
+    cache_k = [np.zeros((s0.n_slots * cap, g.Hkv, g.D), np.float32) for _ in range(L)]      # oracle's, sampled slabs only
+    cache_v = [np.zeros_like(cache_k[0]) for _ in range(L)]
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    L_d, cnt = i32(s0.doc_prefix_len), i32(s0.doc_branch_cnt)
+    depth = torch.zeros(s0.n_slots, dtype=torch.int32, device=dev)
+    alive = torch.ones(s0.n_slots, dtype=torch.uint8, device=dev)
+    meta = B.MetaTables.alloc(g, s0.n_docs, s0.n_slots, s0.total_prefix, dev)
+    q = torch.zeros(s0.n_slots, g.Hq, g.D, dtype=torch.bfloat16, device=dev)
+    kn = torch.zeros(s0.n_slots, g.Hkv, g.D, dtype=torch.bfloat16, device=dev); vn = torch.zeros_like(kn)
+    o = torch.zeros_like(q)
+    steps = int(s0.eos_len.max())
+    checked = 0
+    for t in range(steps):
+        st = synth.loop_step_state(s0, t)
+        if st.n_active == 0:
+            break
+        depth.copy_(torch.from_numpy(st.slot_depth)); alive.copy_(torch.from_numpy(st.slot_alive))
+        B.hpd_build_meta(g, s0.n_docs, s0.n_slots, L_d, cnt, depth, alive, 0, meta)
+        om = capi.build_meta(st.doc_prefix_len, st.doc_branch_cnt, st.slot_depth, st.slot_alive, cap, 0)
+        n = om.n_active
+        assert int(meta.n_active.item()) == n
+        for nm in capi.Meta.TABLES:
+            assert np.array_equal(getattr(meta, nm).cpu().numpy()[: len(getattr(om, nm))], getattr(om, nm)), (t, nm)
+        act = om.active_slot[:n]
+        rows = np.nonzero(np.isin(act, sample))[0]
+        for l in range(L):
+            # the step's activations: the pools read through a permutation that changes with step and layer
+            perm = (act.astype(np.int64) * 7919 + 104729 * (t * L + l + 1)) % s0.n_slots
+            qb, kb, vb = pools["q"][perm], pools["k"][perm], pools["v"][perm]
+            q[:n].copy_(bf(qb)); kn[:n].copy_(bf(kb)); vn[:n].copy_(bf(vb))
+            B.hpd_rope(g, s0.n_slots, meta.n_active, meta.pos_id, q, kn)
+            B.hpd_kv_append(g, s0.n_slots, s0.n_slots, meta.n_active, meta.suffix_off, meta.suffix_len, kn, vn,
+                            suf_k[l], suf_v[l], meta.dev_status)
+            B.hpd_attn_decode(g, s0.n_docs, s0.n_slots, s0.n_slots, s0.total_prefix, q, pre_k[l], pre_v[l], suf_k[l],
+                              suf_v[l], L_d, meta, True, o, None)
+            torch.cuda.synchronize()
+            assert int(meta.dev_status.item()) == 0
+            got_all = synth.bf16_bits_to_f32(runtime.bits_of(o))[:n]
+            assert np.isfinite(got_all).all(), (t, l)
+            if len(rows):
+                fq, fk, fv = (synth.bf16_bits_to_f32(a) for a in (qb, kb, vb))
+                want = capi.decode_step(g, om, st.doc_prefix_len, fq, fk, fv, f_pre[l]["prefix_k"], f_pre[l]["prefix_v"],
+                                        cache_k[l], cache_v[l], rows=rows)
+                d = np.abs(got_all[rows] - want.o)
+                assert d.max() <= MAX_ABS and d.mean() <= MEAN_ABS, (t, l, d.max(), d.mean())
+                dst = (om.suffix_off[:n][rows] + om.suffix_len[:n][rows]).astype(np.int64)
+                cache_k[l][dst] = want.k_rot                     # the append rule of Sec. 4.3.2 for the sampled branches
+                cache_v[l][dst] = fv[rows]
+                checked += len(rows)
+    assert checked == L * int(s0.eos_len[sample].sum())
+    for l in range(L):
+        gk = synth.bf16_bits_to_f32(runtime.bits_of(suf_k[l])).reshape(-1, g.Hkv, g.D)
+        gv = synth.bf16_bits_to_f32(runtime.bits_of(suf_v[l])).reshape(-1, g.Hkv, g.D)
+        written = np.zeros(s0.n_slots * cap, bool)
+        for sl in range(s0.n_slots):
+            written[sl * cap: sl * cap + int(s0.eos_len[sl])] = True
+        assert np.isfinite(gk[written]).all() and np.isfinite(gv[written]).all()
+        assert np.isnan(gk[~written]).all() and np.isnan(gv[~written]).all()      # nothing beyond a value's length
+        for sl in sample:
+            lo, m = sl * cap, int(s0.eos_len[sl])
+            ck = cache_k[l][lo:lo + m]
+            assert np.all(np.abs(gk[lo:lo + m] - ck) <= np.abs(ck) * 2.0 ** -8 + 1e-6)
+            assert np.array_equal(gv[lo:lo + m], cache_v[l][lo:lo + m])

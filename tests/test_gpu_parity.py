@@ -32,6 +32,18 @@ def _ragged(seed, **kw):
     return synth.config_custom("ragged", **d)
 
 
+def _last_slot_full(s):
+    """The last slot alive and one token short of its slab: after the step's append it is full, so the
+    attention's rounded-up K boxes of that branch run past the slab and past the end of the cache tensor."""
+    s.slot_depth[-1] = s.geom.suffix_cap - 1
+    s.slot_alive[-1] = 1
+    return s
+
+
+def _odd_cap(cap, seed):
+    return _last_slot_full(_ragged(seed, cap=cap, depth_hi=cap))
+
+
 STRUCTS = {
     "tiny": lambda: synth.config_tiny(0),
     "main_p2": lambda: synth.config_main(n_prompts=2),
@@ -43,13 +55,29 @@ STRUCTS = {
     "one_group_96": lambda: synth.config_custom("wide", Hq=32, Hkv=8, D=128, theta=500000.0, cap=8,
                                                 prefix_lens=[700], branch_cnts=[96], depth_hi=8, seed=6),
     "few_alive": lambda: _ragged(7, alive_frac=0.1),
-    # more documents than the single-launch table builder takes: the three-kernel path
+    # thousands of documents, many of them empty or without branches: several passes of the block-wide scans
     "many_docs": lambda: synth.config_custom("many", Hq=2, Hkv=1, D=64, theta=10000.0, cap=4,
                                              prefix_lens=[(7 * i) % 23 for i in range(4300)],
                                              branch_cnts=[(i % 3) for i in range(4300)], depth_hi=4, seed=10, alive_frac=0.7),
     # one query head per kv head: 128 branches per unit, four rounds of branch tables, dozens of suffix tiles per unit
     "g1_many_branches": lambda: synth.config_custom("g1", Hq=2, Hkv=2, D=128, theta=10000.0, cap=32,
                                                     prefix_lens=[200, 50, 0], branch_cnts=[200, 130, 70], depth_hi=32, seed=9),
+    # slab sizes that are not a multiple of the four-column padding of packed branch tokens
+    "cap1": lambda: _odd_cap(1, 20),
+    "cap3": lambda: _odd_cap(3, 21),
+    "cap5": lambda: _odd_cap(5, 22),
+    "cap6": lambda: _odd_cap(6, 23),
+    # the shape of the paper's experiments (Appendix B: J = 6 stacked documents, K_max = 30; 16 attributes per category)
+    "paper_j6_n16_k30": lambda: _last_slot_full(synth.config_custom(
+        "paper", Hq=32, Hkv=8, D=128, theta=500000.0, cap=30, prefix_lens=[700, 655, 811, 512, 903, 777],
+        branch_cnts=[16] * 6, depth_hi=30, seed=24)),
+    "paper_gap30": lambda: _last_slot_full(synth.config_custom(
+        "paper_gap", Hq=32, Hkv=8, D=128, theta=500000.0, cap=30, prefix_lens=[300, 0, 411],
+        branch_cnts=[16, 16, 16], depth_hi=30, seed=25, pos_gap=30)),
+    # just below the largest slab the attention kernel indexes (16 branches x 4092 packed columns < 2^16)
+    "cap_limit_g8": lambda: _last_slot_full(synth.config_custom(
+        "caplimit", Hq=8, Hkv=1, D=64, theta=10000.0, cap=4092, prefix_lens=[100], branch_cnts=[16],
+        depth_hi=4092, seed=26)),
     "long_small": lambda: synth.config_custom("long", Hq=32, Hkv=8, D=128, theta=500000.0, cap=32,
                                               prefix_lens=[4096, 1025, 3000], branch_cnts=[12, 12, 12], depth_hi=32, seed=8),
 }
