@@ -150,13 +150,17 @@ int hpd_attn_decode(const hpd_geom* geom /*host*/, int n_docs, int max_rows, int
  * sequence of its own with a private physical copy of [prefix ; branch tokens] (parallel streams
  * as batch elements, Sec. 2; standard batched inference, Sec. 4.3.6).  Same math as
  * hpd_attn_decode on the same tokens, GQA, split-KV.
- *   q [max_rows, Hq, D] bf16 (rotated); dup_k/v [total_tokens, Hkv, D] bf16;
+ *   q [max_rows, Hq, D] bf16 (rotated); dup_k/v [total_tokens, Hkv, D] bf16, total_tokens <= 2^31-1
+ *   (host value: the tensors' extent in token rows; tiles are fetched 16 tokens at a time, and
+ *   whatever a tile holds beyond a sequence's last token -- other sequences' rows, or nothing at the
+ *   end of the tensor -- is masked out and never read past total_tokens);
  *   seq_start [max_rows] int64 first token row of each sequence; seq_len [max_rows] int32;
  *   o [max_rows, Hq, D] bf16; lse nullable.
  * workspace: std_workspace_bytes(); may be NULL when that reports 0.
  */
 size_t std_workspace_bytes(const hpd_geom* geom /*host*/, int max_rows, int max_seq_len);
-int std_attn_decode(const hpd_geom* geom /*host*/, int max_rows, int max_seq_len, const int32_t* n_active,
+int std_attn_decode(const hpd_geom* geom /*host*/, int max_rows, int max_seq_len, long long total_tokens,
+                    const int32_t* n_active,
                     const void* q, const void* dup_k, const void* dup_v,
                     const int64_t* seq_start, const int32_t* seq_len,
                     void* o, float* lse, void* workspace, size_t workspace_bytes, void* stream);
@@ -187,7 +191,8 @@ int std_attn_decode(const hpd_geom* geom /*host*/, int max_rows, int max_seq_len
  *     order them with events.
  */
 size_t std_attn_decode_static_max_bytes(void);
-int std_attn_decode_static(const hpd_geom* geom /*host*/, int max_rows, int max_seq_len, const int32_t* n_active,
+int std_attn_decode_static(const hpd_geom* geom /*host*/, int max_rows, int max_seq_len, long long total_tokens,
+                           const int32_t* n_active,
                            const void* q, const void* dup_k, const void* dup_v,
                            const int64_t* seq_start, const int32_t* seq_len,
                            void* o, float* lse, void* stream);

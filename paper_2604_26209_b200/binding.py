@@ -62,11 +62,11 @@ def load() -> C.CDLL:
         lib.hpd_attn_decode.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int, C.c_int, C.c_int] + [vp] * 12 + \
                                        [C.c_int, vp, vp, vp, C.c_size_t, vp, vp]
         lib.std_attn_decode.restype = C.c_int
-        lib.std_attn_decode.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int] + [vp] * 8 + [vp, C.c_size_t, vp]
+        lib.std_attn_decode.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int, C.c_longlong] + [vp] * 8 + [vp, C.c_size_t, vp]
         lib.std_attn_decode_static_max_bytes.restype = C.c_size_t
         lib.std_attn_decode_static_max_bytes.argtypes = []
         lib.std_attn_decode_static.restype = C.c_int
-        lib.std_attn_decode_static.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int] + [vp] * 8 + [vp]
+        lib.std_attn_decode_static.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int, C.c_longlong] + [vp] * 8 + [vp]
         _lib = lib
     return _lib
 
@@ -170,7 +170,7 @@ def std_attn_decode(geom, max_rows, max_seq_len, n_active, q, dup_k, dup_v, seq_
                     workspace=None):
     g = make_geom(geom)
     wsb = 0 if workspace is None else workspace.numel() * workspace.element_size()
-    rc = load().std_attn_decode(C.byref(g), max_rows, max_seq_len, _ptr(n_active), _ptr(q), _ptr(dup_k), _ptr(dup_v),
+    rc = load().std_attn_decode(C.byref(g), max_rows, max_seq_len, int(dup_k.shape[0]), _ptr(n_active), _ptr(q), _ptr(dup_k), _ptr(dup_v),
                                 _ptr(seq_start), _ptr(seq_len), _ptr(o), _ptr(lse), _ptr(workspace), wsb, _stream())
     _check(rc, "std_attn_decode")
 
@@ -183,7 +183,7 @@ def std_attn_decode_static(geom, max_rows, max_seq_len, n_active, q, dup_k, dup_
     """``std_attn_decode`` with the split-KV scratch inside the library (no workspace, no allocation).
     Returns the status code instead of raising when the problem exceeds the built-in scratch."""
     g = make_geom(geom)
-    rc = load().std_attn_decode_static(C.byref(g), max_rows, max_seq_len, _ptr(n_active), _ptr(q), _ptr(dup_k),
+    rc = load().std_attn_decode_static(C.byref(g), max_rows, max_seq_len, int(dup_k.shape[0]), _ptr(n_active), _ptr(q), _ptr(dup_k),
                                        _ptr(dup_v), _ptr(seq_start), _ptr(seq_len), _ptr(o), _ptr(lse), _stream())
     if rc != -3:
         _check(rc, "std_attn_decode_static")

@@ -173,11 +173,12 @@ int hpd_attn_decode(const hpd_geom* geom, int n_docs, int max_rows, int n_slots,
 
 static int std_splits(const hpd_geom* g, int max_rows, int max_seq_len)
 {
-    // enough warps to fill the machine: split long sequences when the batch is small
-    const long long warps = static_cast<long long>(max_rows) * g->Hkv;
-    const long long target = static_cast<long long>(sm_count()) * 32;
-    if (warps <= 0 || warps >= target) return 1;
-    long long s = (target + warps - 1) / warps;
+    // one persistent CTA per SM takes (sequence, block of 8 kv heads, split) items: split long sequences when the
+    // batch alone gives fewer than two items per SM
+    const long long items = static_cast<long long>(max_rows) * ((g->Hkv + 7) / 8);
+    const long long target = 2ll * sm_count();
+    if (items <= 0 || items >= target) return 1;
+    long long s = (target + items - 1) / items;
     const long long by_len = max_seq_len / 256;       // at least 256 keys per split
     if (s > by_len) s = by_len;
     if (s > 32) s = 32;
@@ -192,29 +193,30 @@ size_t std_workspace_bytes(const hpd_geom* geom, int max_rows, int max_seq_len)
     return sizeof(float) * static_cast<size_t>(max_rows) * geom->Hq * s * (geom->D + 2);
 }
 
-int std_attn_decode(const hpd_geom* geom, int max_rows, int max_seq_len, const int32_t* n_active,
+int std_attn_decode(const hpd_geom* geom, int max_rows, int max_seq_len, long long total_tokens, const int32_t* n_active,
                     const void* q, const void* dup_k, const void* dup_v,
                     const int64_t* seq_start, const int32_t* seq_len,
                     void* o, float* lse, void* workspace, size_t workspace_bytes, void* stream)
 {
     int rc = geom_check(geom);
     if (rc != HPD_OK) return rc;
-    if (max_rows < 0 || max_seq_len < 0) return HPD_E_ARG;
+    if (max_rows < 0 || max_seq_len < 0 || total_tokens < 0) return HPD_E_ARG;
+    if (total_tokens > 0x7fffffffll) return HPD_E_CAPACITY;
     if (max_rows == 0) return HPD_OK;
     if (!n_active || !q || !dup_k || !dup_v || !seq_start || !seq_len || !o) return HPD_E_ARG;
     if (!aligned16(q) || !aligned16(dup_k) || !aligned16(dup_v) || !aligned16(o)) return HPD_E_ARG;
     const int splits = std_splits(geom, max_rows, max_seq_len);
     const size_t need = std_workspace_bytes(geom, max_rows, max_seq_len);
     if (need > 0 && (!workspace || workspace_bytes < need)) return HPD_E_WORKSPACE;
-    SimtArgs s{};
+    StdArgs s{};
     s.g = *geom;
-    s.max_rows = max_rows; s.n_splits = splits; s.n_active = n_active;
+    s.max_rows = max_rows; s.n_splits = splits; s.total_tokens = total_tokens; s.n_active = n_active;
     s.q = static_cast<const __nv_bfloat16*>(q);
-    s.k1 = static_cast<const __nv_bfloat16*>(dup_k); s.v1 = static_cast<const __nv_bfloat16*>(dup_v);
+    s.dup_k = static_cast<const __nv_bfloat16*>(dup_k); s.dup_v = static_cast<const __nv_bfloat16*>(dup_v);
     s.seq_start = seq_start; s.seq_len = seq_len;
     s.o = static_cast<__nv_bfloat16*>(o); s.lse = lse; s.part = static_cast<float*>(workspace);
     s.stream = static_cast<cudaStream_t>(stream);
-    return launch_attn_simt(s);
+    return launch_attn_std(s);
 }
 
 }  // extern "C"

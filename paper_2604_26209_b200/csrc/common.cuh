@@ -100,21 +100,15 @@ struct AttnArgs {
     cudaStream_t stream;
 };
 
-// Scalar (CUDA-core) flash-decode over up to two key segments per row.
-struct SimtArgs {
+// Standard batched decode over private per-sequence K/V copies (std_attn_decode).
+struct StdArgs {
     hpd_geom g;
     int max_rows, n_splits;
+    long long total_tokens;          // token rows of dup_k / dup_v
     const int32_t* n_active;
-    const __nv_bfloat16* q;
-    // segment 1: rows [seg1_start[r], +seg1_len[r]) of k1/v1 (via doc tables when doc_id != nullptr)
-    const __nv_bfloat16 *k1, *v1;
-    const int64_t* seq_start;        // std: per row
-    const int32_t* seq_len;          // std: per row
-    const int32_t *doc_id, *doc_kv_start, *doc_prefix_len;   // hpd: per document
-    // segment 2 (hpd only): rows [suffix_off[r], +suffix_len[r]+suffix_extra) of k2/v2
-    const __nv_bfloat16 *k2, *v2;
-    const int32_t *suffix_off, *suffix_len;
-    int suffix_extra;
+    const __nv_bfloat16 *q, *dup_k, *dup_v;
+    const int64_t* seq_start;        // per row: first token row of the sequence
+    const int32_t* seq_len;          // per row
     __nv_bfloat16* o;
     float* lse;
     float* part;                     // n_splits > 1: [max_rows, Hq, n_splits, D+2]
@@ -132,7 +126,7 @@ int launch_rope(const hpd_geom& g, int max_rows, const int32_t* n_active, const 
 int launch_kv_append(const hpd_geom& g, int max_rows, int n_slots, const int32_t* n_active, const int32_t* suffix_off,
                      const int32_t* suffix_len, const __nv_bfloat16* k_new, const __nv_bfloat16* v_new,
                      __nv_bfloat16* suffix_k, __nv_bfloat16* suffix_v, int32_t* dev_status, cudaStream_t stream);
-int launch_attn_simt(const SimtArgs& a);
+int launch_attn_std(const StdArgs& a);         // TMA ring + warp-level tensor-core instructions
 int launch_attn_tc(const AttnArgs& a);       // tcgen05 / TMA kernel
 
 // ---------------------------------------------------------------------------------------------

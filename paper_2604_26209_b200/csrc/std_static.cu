@@ -47,7 +47,7 @@ extern "C" {
 
 size_t std_attn_decode_static_max_bytes(void) { return kScratchBytes; }
 
-int std_attn_decode_static(const hpd_geom* geom, int max_rows, int max_seq_len, const int32_t* n_active,
+int std_attn_decode_static(const hpd_geom* geom, int max_rows, int max_seq_len, long long total_tokens, const int32_t* n_active,
                            const void* q, const void* dup_k, const void* dup_v,
                            const int64_t* seq_start, const int32_t* seq_len,
                            void* o, float* lse, void* stream)
@@ -62,7 +62,7 @@ int std_attn_decode_static(const hpd_geom* geom, int max_rows, int max_seq_len, 
     rc = scratch_for_current_device(&scratch);
     if (rc != HPD_OK) return rc;
     // Every partial that the merge reads is written by the same call first, so nothing has to be cleared.
-    return std_attn_decode(geom, max_rows, max_seq_len, n_active, q, dup_k, dup_v, seq_start, seq_len, o, lse,
+    return std_attn_decode(geom, max_rows, max_seq_len, total_tokens, n_active, q, dup_k, dup_v, seq_start, seq_len, o, lse,
                            scratch, kScratchBytes, stream);
 }
 

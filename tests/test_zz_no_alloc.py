@@ -74,13 +74,20 @@ def test_static_scratch_rejects_oversized_problem():
         pytest.skip("no CUDA device")
     from paper_2604_26209_b200 import binding
     s, tb, db, dup = _batch(23)
-    # the split count, and with it the scratch a problem needs, depends on the GPU's SM count: search for a row count
-    # whose need exceeds the built-in array instead of assuming one
+    # the split count, and with it the scratch a problem needs, depends on the GPU's SM count and on the number of
+    # heads: search for a problem whose need exceeds the built-in array instead of assuming one
+    from dataclasses import replace
     seq, limit = 4096, binding.std_attn_decode_static_max_bytes()
-    rows = next((r for r in range(64, 1 << 16, 64) if binding.std_workspace_bytes(s.geom, r, seq) > limit), None)
-    if rows is None:
+    found = None
+    for geom in (s.geom, replace(s.geom, Hq=512, Hkv=64)):
+        rows = next((r for r in range(1, 2048) if binding.std_workspace_bytes(geom, r, seq) > limit), None)
+        if rows is not None:
+            found = (geom, rows)
+            break
+    if found is None:
         pytest.skip("no problem size on this GPU needs more scratch than the built-in array")
-    rc = binding.std_attn_decode_static(s.geom, rows, seq, dup.n_active, db.q, dup.dup_k, dup.dup_v, dup.seq_start,
+    geom, rows = found
+    rc = binding.std_attn_decode_static(geom, rows, seq, dup.n_active, db.q, dup.dup_k, dup.dup_v, dup.seq_start,
                                         dup.seq_len, dup.o, dup.lse)
     assert rc == -3                             # HPD_E_WORKSPACE, nothing launched
     torch.cuda.synchronize()
