@@ -7,8 +7,10 @@ x 512 prefix tokens x 24 branches, depths uniform in [0,16)).  Prints ONE JSON l
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload main|long]
 
-N > 1 is launched by torchrun, one rank per GPU; prompts are independent, so every rank runs its own
-batch of the same shape (different seed) with no collective on the data path (weak scaling).
+N > 1: one rank per GPU, started by torchrun or, when no rank environment is present, by this script
+itself.  Prompts are independent, so the global prompt list (N x the single-GPU batch) is split into
+contiguous shards, every rank decodes its own shard, and nothing crosses NVLink on the data path (weak
+scaling); only the timing scalars are reduced.
 ``--impl reference`` times the CPU oracle, as it stands, on a bounded sample of the same workload.
 """
 from __future__ import annotations
@@ -32,14 +34,30 @@ METRIC = "branch_tokens_per_s_per_decode_step"
 UNIT = "branch-tokens/s"
 
 
-def make_structure(workload: str, seed: int):
+def workload_prompts(workload: str) -> int:
+    """Prompts of the single-GPU batch of a workload."""
     if workload == "main":
-        return synth.config_main(n_prompts=64, seed=seed)
+        return 64
     if workload == "long":
-        return synth.config_long(n_prompts=32, seed=seed)
+        return 32
     if workload.startswith("main_p"):
-        return synth.config_main(n_prompts=int(workload[6:]), seed=seed)
+        return int(workload[6:])
     raise SystemExit(f"unknown workload {workload}")
+
+
+def rank_structure(workload: str, world: int, rank: int):
+    """The shard of the global prompt list that rank ``rank`` of ``world`` decodes (no GPU needed).
+
+    The global batch has ``world`` x the single-GPU prompts; ``synth.shard_prompts`` gives each rank a contiguous
+    range of prompt indices; the rank's structure is drawn with the index of its first prompt as seed, so rank 0 of
+    a one-rank run is the single-GPU workload itself.  Returns (structure, range of global prompt indices)."""
+    per_gpu = workload_prompts(workload)
+    mine = synth.shard_prompts(per_gpu * world, world, rank)
+    if workload == "long":
+        s = synth.config_long(n_prompts=len(mine), seed=mine.start)
+    else:
+        s = synth.config_main(n_prompts=len(mine), seed=mine.start)
+    return s, mine
 
 
 def algorithmic_bytes(s) -> dict:
@@ -69,43 +87,55 @@ def measured_peaks() -> dict:
 
 
 class ClockSampler:
-    """nvidia-smi clock/throttle samples during the timed region (read-only query)."""
+    """nvidia-smi clock/throttle samples (read-only query), time-stamped so that only those taken inside the timed
+    regions are summarised."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int):
-        self.index, self.lines, self.proc = index, [], None
+    def __init__(self, index: int, period_ms: int = 50):
+        self.index, self.period_ms, self.lines, self.proc, self.windows = index, period_ms, [], None, []
 
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+                                          "-i", str(self.index), "-lms", str(self.period_ms)],
+                                         stdout=subprocess.PIPE, text=True)
             threading.Thread(target=self._pump, daemon=True).start()
         except Exception:
             self.proc = None
 
     def _pump(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.time(), line.strip()))
+
+    def window(self, t0: float, t1: float):
+        """Mark [t0, t1] (time.time()) as a timed region."""
+        self.windows.append((t0, t1))
 
     def stop(self) -> dict:
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(2 * self.period_ms * 1e-3)
         self.proc.terminate()
-        sm, mx, reasons = [], [], set()
-        for ln in self.lines:
+        sm, mx, pw, reasons, n_all = [], [], [], set(), 0
+        for ts, ln in self.lines:
             f = [x.strip() for x in ln.split(",")]
             if len(f) < 9:
                 continue
+            n_all += 1
+            if self.windows and not any(t0 <= ts <= t1 + self.period_ms * 1e-3 for t0, t1 in self.windows):
+                continue
             try:
-                sm.append(float(f[1])); mx.append(float(f[2]))
+                sm.append(float(f[1])); mx.append(float(f[2])); pw.append(float(f[3]))
             except ValueError:
                 continue
             for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "samples_total": n_all,
+                "power_w_max": max(pw) if pw else None,
+                "note": "samples taken inside the timed regions (graph replay, direct calls, end to end)"}
 
 
 def time_oracle_sample(s, tb, budget_rows: int, n_threads: int = 0):
@@ -128,7 +158,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    s = make_structure(args.workload, 0)
+    s, _ = rank_structure(args.workload, 1, 0)
     tb = synth.make_tensors(s)
     rows_per_step = 256
     for _ in range(args.warmup):
@@ -151,10 +181,24 @@ def run_reference(args):
     }))
 
 
+def block_stats(ms) -> dict:
+    a = np.asarray(ms, dtype=np.float64)
+    return {"blocks": int(a.size), "median_ms": float(np.median(a)), "min_ms": float(a.min()), "max_ms": float(a.max()),
+            "p10_ms": float(np.percentile(a, 10)), "p90_ms": float(np.percentile(a, 90))}
+
+
+def agree_block_count(first_block_ms: float, target_ms: float, reduce_max) -> int:
+    """How many K-step blocks to time so that about ``target_ms`` of device time is covered; every rank gets the
+    same count (the slowest rank's first block decides)."""
+    t = max(reduce_max(first_block_ms), 1e-3)
+    return int(min(max(np.ceil(target_ms / t), 3), 5000))
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
     from paper_2604_26209_b200 import runtime, binding
+    from paper_2604_26209_b200.dist import reduce_timing
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -166,7 +210,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     binding.load()
 
-    s = make_structure(args.workload, seed=rank)          # every rank: its own prompts, same shape
+    s, my_prompts = rank_structure(args.workload, world, rank)      # this rank's shard of the global prompt list
     tb = synth.make_tensors(s)
     db = runtime.DeviceBatch(s, tb)
     db.build_meta()
@@ -179,6 +223,7 @@ def run_ours(args):
     assert ab["n_active"] == n
 
     stream = torch.cuda.current_stream()
+    K = args.steps
 
     def barrier():
         torch.cuda.synchronize()
@@ -186,50 +231,73 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident timing ---------------------------------------------------------------------------
-    for _ in range(args.warmup):
-        db.step(with_meta=True)
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    def reduce_max(x: float) -> float:
+        return reduce_timing([x], 0, device="cuda")[0][0]
+
+    def time_block(fn) -> float:
+        """Exactly K steps between two events, a barrier and a synchronize on both sides."""
+        barrier()
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(K):
+            fn()
+        e1.record(stream)
+        barrier()
+        return e0.elapsed_time(e1)
+
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-        time.sleep(0.3)
-    barrier()
-    t_all0 = torch.cuda.Event(enable_timing=True); t_all1 = torch.cuda.Event(enable_timing=True)
-    t_all0.record(stream)
-    for i in range(args.steps):
-        ev[i][0].record(stream)
-        db.build_meta(); db.rope(); db.kv_append()
-        ev[i][1].record(stream)
-        db.attn(True)
-        ev[i][2].record(stream)
-    t_all1.record(stream)
-    barrier()
-    clocks = sampler.stop() if rank == 0 else None
-    ms_total = t_all0.elapsed_time(t_all1)
-    ms_attn = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
-    ms_pre = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
+        time.sleep(0.2)
+
+    # ---- direct C-ABI calls, one per operation, CUDA events between them: per-kernel breakdown --------------------
+    for _ in range(args.warmup):
+        db.step(with_meta=True, fused=not args.unfused)
+
+    def direct_block():
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+        barrier()
+        for i in range(K):
+            ev[i][0].record(stream)
+            db.build_meta()
+            if args.unfused:
+                db.rope(); db.kv_append()
+            else:
+                db.rope_append()
+            ev[i][1].record(stream)
+            db.attn(True)
+            ev[i][2].record(stream)
+        barrier()
+        return (ev[0][0].elapsed_time(ev[-1][2]), float(np.mean([e[1].elapsed_time(e[2]) for e in ev])),
+                float(np.mean([e[0].elapsed_time(e[1]) for e in ev])))
+
+    first = direct_block()
+    n_direct = agree_block_count(first[0], args.min_ms * 0.4, reduce_max)
+    t_w0 = time.time()
+    direct = [direct_block() for _ in range(n_direct)]
+    sampler.window(t_w0, time.time())
+    ms_total_blocks = [d[0] for d in direct]
+    ms_attn = float(np.median([d[1] for d in direct]))
+    ms_pre = float(np.median([d[2] for d in direct]))
+    attn_stats = block_stats([d[1] for d in direct])
     status = db.status()
 
-    # ---- the same step replayed from a CUDA graph (extra information: launch-bound small batches) ---------
-    ms_graph = None
+    # ---- the same step replayed from a CUDA graph: the headline ----------------------------------------------------
+    graph_blocks = None
     if not args.no_graph:
         barrier()
-        g = db.capture_step(with_meta=True)
+        g = db.capture_step(with_meta=True, fused=not args.unfused)
         for _ in range(3):
             g.replay()
-        barrier()
-        g0 = torch.cuda.Event(enable_timing=True); g1 = torch.cuda.Event(enable_timing=True)
-        g0.record(stream)
-        for _ in range(args.steps):
-            g.replay()
-        g1.record(stream)
-        barrier()
-        ms_graph = g0.elapsed_time(g1)
+        first_g = time_block(g.replay)
+        n_graph = agree_block_count(first_g, args.min_ms, reduce_max)
+        t_w0 = time.time()
+        graph_blocks = [time_block(g.replay) for _ in range(n_graph)]
+        sampler.window(t_w0, time.time())
         if db.status() != 0:
             status = db.status()
 
-    # ---- end to end: host buffers in, host result out, through the same calls ------------------------------
+    # ---- end to end: host buffers in, host result out, through the same calls ------------------------------------
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
     hq, hk, hv = pin(tb["q"][act]), pin(tb["k_new"][act]), pin(tb["v_new"][act])
     h_depth = torch.from_numpy(s.slot_depth.copy()).pin_memory()
@@ -244,34 +312,34 @@ def run_ours(args):
         db.q[:n].view(torch.int16).copy_(hq, non_blocking=True)
         db.k_new[:n].view(torch.int16).copy_(hk, non_blocking=True)
         db.v_new[:n].view(torch.int16).copy_(hv, non_blocking=True)
-        db.step(with_meta=True)
+        db.step(with_meta=True, fused=not args.unfused)
         h_o.copy_(db.o[:n].view(torch.int16), non_blocking=True)
 
-    e2e_steps = max(3, min(args.steps, 20))
     for _ in range(3):
         e2e_step()
-    barrier()
-    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(e2e_steps):
-        e2e_step()
-    e1.record(stream)
-    barrier()
-    ms_e2e = e0.elapsed_time(e1)
+    first_e = time_block(e2e_step)
+    n_e2e = agree_block_count(first_e, args.min_ms * 0.3, reduce_max)
+    t_w0 = time.time()
+    e2e_blocks = [time_block(e2e_step) for _ in range(n_e2e)]
+    sampler.window(t_w0, time.time())
+    clocks = sampler.stop() if rank == 0 else None
 
-    # ---- max over ranks (time), sum over ranks (rows) ----------------------------------------------------------
-    from paper_2604_26209_b200.dist import reduce_timing
-    (ms_total, ms_e2e, ms_attn_max, ms_graph_max), tok_all = reduce_timing(
-        [ms_total, ms_e2e, ms_attn, ms_graph if ms_graph is not None else 0.0], n, device="cuda")
+    # ---- max over ranks of every block time, sum over ranks of the rows -------------------------------------------
+    head_blocks = graph_blocks if graph_blocks is not None else ms_total_blocks
+    head_max, tok_all = reduce_timing(head_blocks, n, device="cuda")
+    direct_max, _ = reduce_timing(ms_total_blocks, 0, device="cuda")
+    e2e_max, _ = reduce_timing(e2e_blocks, 0, device="cuda")
+    (ms_attn_max,), _ = reduce_timing([ms_attn], 0, device="cuda")
 
     if rank == 0:
         peaks = measured_peaks()
-        # Headline: the K steps replayed from a CUDA graph (the same seven kernels per step, launched back to back by the
-        # GPU instead of one host call each); the direct-call pass gives the per-kernel breakdown and is reported too.
-        value_direct = tok_all * args.steps / (ms_total * 1e-3)
-        ms_head = ms_graph_max if ms_graph is not None else ms_total
-        value = tok_all * args.steps / (ms_head * 1e-3)
-        e2e_val = tok_all * e2e_steps / (ms_e2e * 1e-3)
+        # Headline: K steps replayed from a CUDA graph (the same kernels per step, launched back to back by the GPU
+        # instead of one host call each), median over the timed K-step blocks of the slowest rank's time.
+        hs, ds, es = block_stats(head_max), block_stats(direct_max), block_stats(e2e_max)
+        ms_head = hs["median_ms"]
+        value = tok_all * K / (ms_head * 1e-3)
+        value_direct = tok_all * K / (ds["median_ms"] * 1e-3)
+        e2e_val = tok_all * K / (es["median_ms"] * 1e-3)
         ach = ab["attn"] / (ms_attn * 1e-3) / 1e9
         tflops = ab["flops"] / (ms_attn * 1e-3) / 1e12
         cpu = None
@@ -293,56 +361,90 @@ def run_ours(args):
                         + s.slot_depth[s.slot_alive.astype(bool)] + 1).sum()) * row_b
             rows_std = n if need < 0.6 * free_b else max(1, int(n * 0.6 * free_b / need))
             dup = runtime.DupBatch(db, include_new=True, rows=rows_std)
-            for _ in range(2):
-                dup.attn(db.q)
-            c0 = torch.cuda.Event(enable_timing=True); c1 = torch.cuda.Event(enable_timing=True)
-            torch.cuda.synchronize()
-            c0.record(stream)
             for _ in range(3):
                 dup.attn(db.q)
-            c1.record(stream)
-            torch.cuda.synchronize()
-            ms_std = c0.elapsed_time(c1) / 3 * (n / dup.n)          # linear in rows: no sharing between sequences
+            reps, t_std = 5, []
+            for _ in range(7):
+                c0 = torch.cuda.Event(enable_timing=True); c1 = torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                c0.record(stream)
+                for _ in range(reps):
+                    dup.attn(db.q)
+                c1.record(stream)
+                torch.cuda.synchronize()
+                t_std.append(c0.elapsed_time(c1) / reps)
+            ms_std = float(np.median(t_std)) * (n / dup.n)          # linear in rows: no sharing between sequences
             std_bytes = dup.total_tokens * row_b * (n / dup.n) + ab["qo"]
             comparison = {"kernel": "std_attn_decode (duplicated prefix)", "ms_per_launch": ms_std,
                           "rows_timed": dup.n, "rows_total": n,
                           "hbm_frac_of_measured": std_bytes / (ms_std * 1e-3) / 1e9 / peaks["hbm_gbs"],
                           "algorithmic_bytes": int(std_bytes), "bytes_ratio_std_over_hpd": std_bytes / ab["attn"],
-                          "speedup_hpd_over_std": ms_std / ms_attn}
+                          "speedup_hpd_over_std": ms_std / ms_attn,
+                          "note": "the speedup is bounded by the byte ratio; both kernels stream at their own fraction of HBM"}
             del dup
         traffic = None
         tp = os.path.join(ROOT, "profiles", "traffic.json")
         if os.path.exists(tp):
             traffic = json.load(open(tp)).get(f"hpd_attn_decode:{s.name}")
-        launches_per_step = 3 + 1 + 1 + 2                  # table kernels, rope, append, attention + merge
+        launches_per_step = 3 + (2 if args.unfused else 1) + 2      # table kernels, rope/append, attention + merge
+        n_steps_timed = K * (len(head_blocks) + len(ms_total_blocks) + len(e2e_blocks))
         out = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms_head / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
+            "ms_per_step": ms_head / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": s.name, "prompts_per_gpu": s.n_prompts, "branches_per_prompt": 96,
-                       "docs_per_prompt": s.docs_per_prompt, "n_active_per_gpu": n, "geometry": "Hq32/Hkv8/D128",
-                       "layers": 1, "l2": f"inputs larger than L2 ({ab['attn'] / 1e6:.0f} MB touched per step vs 126 MB L2); no flush",
-                       "attn_impl": os.environ.get("HPD_ATTN_IMPL", "default")},
+            "config": {"workload": s.name, "prompts_per_gpu": s.n_prompts, "global_prompts": s.n_prompts * world,
+                       "branches_per_prompt": 96, "docs_per_prompt": s.docs_per_prompt, "n_active_per_gpu": n,
+                       "geometry": "Hq32/Hkv8/D128", "layers": 1,
+                       "l2": f"inputs larger than L2 ({ab['attn'] / 1e6:.0f} MB touched per step vs 126 MB L2); no flush",
+                       "rope_append": "two launches" if args.unfused else "one launch (hpd_rope_append)"},
+            "timing": {"what": f"blocks of exactly {K} steps, each between a barrier + synchronize; value = median block",
+                       "headline": hs, "direct_calls": ds, "e2e": es, "attn_launch_ms_per_block_mean": attn_stats},
             "clocks": clocks,
             "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-                    "ms_per_step": ms_e2e / e2e_steps, "steps": e2e_steps},
-            "gpu_launches": launches_per_step * args.steps,
+                    "ms_per_step": es["median_ms"] / K, "steps": K},
+            "gpu_launches": launches_per_step * K,
+            "gpu_launches_all_timed_regions": launches_per_step * n_steps_timed,
             "roofline": {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": ach / peaks["hbm_gbs"], "traffic": traffic, "kernel": "hpd_attn_decode",
                          "peak_source": peaks["source"], "ms_per_launch": ms_attn, "algorithmic_bytes": ab["attn"],
                          "frac_of_nominal_8TBs": ach / 8000.0, "tensor_tflops_algorithmic": tflops,
                          "tensor_frac_of_measured_bf16": tflops / peaks["bf16_tflops"]},
             "breakdown_ms": {"meta_rope_append": ms_pre, "attn": ms_attn},
-            "launch": ("cuda graph replay of the step (captured once from the C-ABI calls)" if ms_graph is not None
+            "launch": ("cuda graph replay of the step (captured once from the C-ABI calls)" if graph_blocks is not None
                        else "one C-ABI call per kernel group"),
-            "direct_calls": {"ms_per_step": ms_total / args.steps, "value": value_direct, "unit": UNIT,
+            "direct_calls": {"ms_per_step": ds["median_ms"] / K, "value": value_direct, "unit": UNIT,
                              "note": "the same K steps as one C-ABI call per operation with CUDA events between them; "
                                      "source of breakdown_ms and of the roofline's launch time"},
             "cpu_baseline": cpu, "comparison": comparison, "dev_status": status,
         }
-        print(json.dumps(out))
+        print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def spawn_ranks(args) -> int:
+    """``--gpus N`` without a rank environment: start one process per GPU (the environment torchrun would give them),
+    wait for all, pass rank 0's JSON line through."""
+    import socket
+    import torch
+    have = torch.cuda.device_count()
+    world = min(args.gpus, have) if have > 0 else 0
+    if world < 1:
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    if world < args.gpus:
+        sys.stderr.write(f"bench.py: {args.gpus} GPUs asked for, {have} visible: running {world} ranks\n")
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    procs = []
+    for r in range(world):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(world), LOCAL_WORLD_SIZE=str(world),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__), *sys.argv[1:]], env=env))
+    rc = 0
+    for p in procs:
+        rc = max(rc, p.wait())
+    return rc
 
 
 def run_loop(args):
@@ -432,7 +534,7 @@ def run_loop(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="main")
@@ -441,6 +543,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-comparison", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay leg")
+    ap.add_argument("--unfused", action="store_true", help="hpd_rope and hpd_kv_append as two launches instead of hpd_rope_append")
+    ap.add_argument("--min-ms", type=float, default=1000.0, help="device time to cover with timed K-step blocks")
     ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--loop-prompts", type=int, default=64)
     args = ap.parse_args()
@@ -450,6 +554,8 @@ def main():
         run_loop(args)
     elif args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
     else:
         run_ours(args)
 

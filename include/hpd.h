@@ -124,6 +124,18 @@ int hpd_kv_append(const hpd_geom* geom /*host*/, int max_rows, int n_slots, cons
                   int32_t* dev_status, void* stream);
 
 /*
+ * hpd_rope_append -- hpd_rope followed by hpd_kv_append in ONE launch (Sec. 4.3.1-4.3.2: the new token
+ * is rotated at its assigned position ID and appended to the cache).  q and k_new are rotated in place
+ * and the rotated key and the value go to row suffix_off[r] + suffix_len[r] of the branch cache; every
+ * output bit equals that of the two separate calls, as do the status bits (a full slab still gets its q
+ * and k rotated, no cache write, HPD_S_OVERFLOW).  Arguments as in the two calls.
+ */
+int hpd_rope_append(const hpd_geom* geom /*host*/, int max_rows, int n_slots, const int32_t* n_active,
+                    const int32_t* pos_id, const int32_t* suffix_off, const int32_t* suffix_len,
+                    void* q, void* k_new, const void* v_new, void* suffix_k, void* suffix_v,
+                    int32_t* dev_status, void* stream);
+
+/*
  * hpd_attn_decode -- the HPD decode attention (Eq. 5-6; Sec. 4.3.3).  For row r (document d,
  * slot s) and q head h:   o = softmax(sm_scale * q . [K_prefix(d) ; K_suffix(s)]^T) [V_prefix(d) ; V_suffix(s)]
  * over the document's L_d prefix tokens and the branch's own cached tokens.  The prefix of a

@@ -18,7 +18,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libhpd.so")
 
 EXPORTS = ("hpd_strerror", "hpd_last_cuda_error", "hpd_workspace_bytes", "hpd_build_meta", "hpd_rope",
-           "hpd_kv_append", "hpd_attn_decode", "std_workspace_bytes", "std_attn_decode",
+           "hpd_kv_append", "hpd_rope_append", "hpd_attn_decode", "std_workspace_bytes", "std_attn_decode",
            "std_attn_decode_static_max_bytes", "std_attn_decode_static")
 
 HPD_S_OVERFLOW, HPD_S_BAD_TABLE, HPD_S_TIMEOUT = 1, 2, 4
@@ -58,6 +58,8 @@ def load() -> C.CDLL:
         lib.hpd_rope.argtypes = [C.POINTER(HpdGeom), C.c_int, vp, vp, vp, vp, vp]
         lib.hpd_kv_append.restype = C.c_int
         lib.hpd_kv_append.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int] + [vp] * 9
+        lib.hpd_rope_append.restype = C.c_int
+        lib.hpd_rope_append.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int] + [vp] * 11
         lib.hpd_attn_decode.restype = C.c_int
         lib.hpd_attn_decode.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int, C.c_int, C.c_int] + [vp] * 12 + \
                                        [C.c_int, vp, vp, vp, C.c_size_t, vp, vp]
@@ -153,6 +155,15 @@ def hpd_kv_append(geom, max_rows, n_slots, n_active, suffix_off, suffix_len, k_n
     rc = load().hpd_kv_append(C.byref(g), max_rows, n_slots, _ptr(n_active), _ptr(suffix_off), _ptr(suffix_len),
                               _ptr(k_new), _ptr(v_new), _ptr(suffix_k), _ptr(suffix_v), _ptr(dev_status), _stream())
     _check(rc, "hpd_kv_append")
+
+
+def hpd_rope_append(geom, max_rows, n_slots, n_active, pos_id, suffix_off, suffix_len, q, k_new, v_new, suffix_k, suffix_v,
+                    dev_status):
+    g = make_geom(geom)
+    rc = load().hpd_rope_append(C.byref(g), max_rows, n_slots, _ptr(n_active), _ptr(pos_id), _ptr(suffix_off),
+                                _ptr(suffix_len), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(suffix_k), _ptr(suffix_v),
+                                _ptr(dev_status), _stream())
+    _check(rc, "hpd_rope_append")
 
 
 def hpd_attn_decode(geom, n_docs, max_rows, n_slots, total_prefix_tokens, q, prefix_k, prefix_v, suffix_k, suffix_v,

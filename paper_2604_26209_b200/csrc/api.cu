@@ -130,6 +130,22 @@ int hpd_kv_append(const hpd_geom* geom, int max_rows, int n_slots, const int32_t
                             static_cast<cudaStream_t>(stream));
 }
 
+int hpd_rope_append(const hpd_geom* geom, int max_rows, int n_slots, const int32_t* n_active, const int32_t* pos_id,
+                    const int32_t* suffix_off, const int32_t* suffix_len, void* q, void* k_new, const void* v_new,
+                    void* suffix_k, void* suffix_v, int32_t* dev_status, void* stream)
+{
+    int rc = geom_check(geom);
+    if (rc != HPD_OK) return rc;
+    if (max_rows < 0 || n_slots < 0) return HPD_E_ARG;
+    if (max_rows == 0) return HPD_OK;
+    if (!n_active || !pos_id || !suffix_off || !suffix_len || !q || !k_new || !v_new || !suffix_k || !suffix_v) return HPD_E_ARG;
+    if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(suffix_k) || !aligned16(suffix_v)) return HPD_E_ARG;
+    return launch_rope_append(*geom, max_rows, n_slots, n_active, pos_id, suffix_off, suffix_len,
+                              static_cast<__nv_bfloat16*>(q), static_cast<__nv_bfloat16*>(k_new),
+                              static_cast<const __nv_bfloat16*>(v_new), static_cast<__nv_bfloat16*>(suffix_k),
+                              static_cast<__nv_bfloat16*>(suffix_v), dev_status, static_cast<cudaStream_t>(stream));
+}
+
 int hpd_attn_decode(const hpd_geom* geom, int n_docs, int max_rows, int n_slots, int total_prefix_tokens,
                     const void* q, const void* prefix_k, const void* prefix_v,
                     const void* suffix_k, const void* suffix_v,

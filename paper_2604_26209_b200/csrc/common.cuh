@@ -126,6 +126,10 @@ int launch_rope(const hpd_geom& g, int max_rows, const int32_t* n_active, const 
 int launch_kv_append(const hpd_geom& g, int max_rows, int n_slots, const int32_t* n_active, const int32_t* suffix_off,
                      const int32_t* suffix_len, const __nv_bfloat16* k_new, const __nv_bfloat16* v_new,
                      __nv_bfloat16* suffix_k, __nv_bfloat16* suffix_v, int32_t* dev_status, cudaStream_t stream);
+int launch_rope_append(const hpd_geom& g, int max_rows, int n_slots, const int32_t* n_active, const int32_t* pos_id,
+                       const int32_t* suffix_off, const int32_t* suffix_len, __nv_bfloat16* q, __nv_bfloat16* k_new,
+                       const __nv_bfloat16* v_new, __nv_bfloat16* suffix_k, __nv_bfloat16* suffix_v, int32_t* dev_status,
+                       cudaStream_t stream);
 int launch_attn_std(const StdArgs& a);         // TMA ring + warp-level tensor-core instructions
 int launch_attn_tc(const AttnArgs& a);       // tcgen05 / TMA kernel
 

@@ -1,7 +1,10 @@
-// hpd_rope and hpd_kv_append: the two streaming kernels around the attention.
+// hpd_rope, hpd_kv_append and their fusion hpd_rope_append: the streaming kernels around the attention.
 //
-// Both are pure HBM streaming (read + write of the step's new q/k/v rows); one CTA per row,
+// All are pure HBM streaming (read + write of the step's new q/k/v rows); one CTA per row,
 // 16-byte accesses, grid sized by max_rows with an early exit on the device-side row count.
+// The fused kernel rotates q and k in place, and while a rotated key chunk is still in registers also
+// stores it to the row's slot in the branch cache, then copies the value row there: one launch and one
+// read of k instead of two, the same bits as the two separate calls.
 #include "common.cuh"
 
 namespace hpd {
@@ -14,10 +17,20 @@ constexpr int kRopeThreads = 256;
 // thousands of radians, where an fp32 product pos * inv_freq already loses ~1e-4 rad), kept in
 // shared memory as fp32, and applied to all Hq + Hkv heads: each thread rotates 8 pairs at a time
 // from one 16-byte load of the low half and one of the high half.
-template <int D>
+struct AppendDst {                                   // fused kernel only: where the row's key and value go
+    int32_t suffix_cap;
+    int64_t cache_rows;
+    const int32_t *suffix_off, *suffix_len;
+    const __nv_bfloat16* v_new;
+    __nv_bfloat16 *suffix_k, *suffix_v;
+    int32_t* dev_status;
+};
+
+template <int D, bool FUSED>
 __global__ void __launch_bounds__(kRopeThreads)
 rope_kernel(int Hq, int Hkv, double neg_log2_theta_2_over_d, const int32_t* __restrict__ n_active,
-            const int32_t* __restrict__ pos_id, __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ k_new)
+            const int32_t* __restrict__ pos_id, __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ k_new,
+            const AppendDst ad)
 {
     constexpr int HALF = D / 2;
     constexpr int CHUNKS = HALF / 8;                 // 16-byte chunks per half
@@ -25,6 +38,19 @@ rope_kernel(int Hq, int Hkv, double neg_log2_theta_2_over_d, const int32_t* __re
     const int r = blockIdx.x;
     if (r >= *n_active) return;
     const int pos = pos_id[r];
+    // destination row in the branch cache (-1: slab full or table entry out of range -> status bit, no write)
+    int64_t dst_row = -1;
+    if constexpr (FUSED) {
+        const int len = ad.suffix_len[r];
+        const int64_t off = ad.suffix_off[r];
+        if (len >= ad.suffix_cap || len < 0) {
+            if (threadIdx.x == 0 && ad.dev_status) atomicOr(ad.dev_status, HPD_S_OVERFLOW);
+        } else if (off < 0 || off + len >= ad.cache_rows) {
+            if (threadIdx.x == 0 && ad.dev_status) atomicOr(ad.dev_status, HPD_S_BAD_TABLE);
+        } else {
+            dst_row = off + len;
+        }
+    }
     if (threadIdx.x < HALF) {
         const double inv_freq = exp2(neg_log2_theta_2_over_d * static_cast<double>(threadIdx.x));
         double s, c;
@@ -34,7 +60,18 @@ rope_kernel(int Hq, int Hkv, double neg_log2_theta_2_over_d, const int32_t* __re
     }
     __syncthreads();
     const int items = (Hq + Hkv) * CHUNKS;
-    for (int it = threadIdx.x; it < items; it += kRopeThreads) {
+    // fused: the value row's 16-byte pieces are further items, so the threads left over by the rotation copy them
+    const int row_u4 = Hkv * D / 8;
+    const int all_items = (FUSED && dst_row >= 0) ? items + row_u4 : items;
+    for (int it = threadIdx.x; it < all_items; it += kRopeThreads) {
+        if constexpr (FUSED) {
+            if (it >= items) {
+                const int i = it - items;
+                reinterpret_cast<uint4*>(ad.suffix_v)[dst_row * row_u4 + i] =
+                    reinterpret_cast<const uint4*>(ad.v_new)[static_cast<int64_t>(r) * row_u4 + i];
+                continue;
+            }
+        }
         const int head = it / CHUNKS, ch = it % CHUNKS;
         __nv_bfloat16* base = head < Hq ? q + (static_cast<int64_t>(r) * Hq + head) * D
                                         : k_new + (static_cast<int64_t>(r) * Hkv + (head - Hq)) * D;
@@ -54,6 +91,13 @@ rope_kernel(int Hq, int Hkv, double neg_log2_theta_2_over_d, const int32_t* __re
         }
         *plo = lo;
         *phi = hi;
+        if constexpr (FUSED) {
+            if (head >= Hq && dst_row >= 0) {
+                uint4* cd = reinterpret_cast<uint4*>(ad.suffix_k + (dst_row * Hkv + (head - Hq)) * D);
+                cd[ch] = lo;
+                cd[CHUNKS + ch] = hi;
+            }
+        }
     }
 }
 
@@ -96,10 +140,28 @@ int launch_rope(const hpd_geom& g, int max_rows, const int32_t* n_active, const 
 {
     if (max_rows <= 0) return HPD_OK;
     const double c = -2.0 * log2(static_cast<double>(g.rope_theta)) / static_cast<double>(g.D);
+    const AppendDst none{};
     if (g.D == 128)
-        rope_kernel<128><<<max_rows, kRopeThreads, 0, stream>>>(g.Hq, g.Hkv, c, n_active, pos_id, q, k_new);
+        rope_kernel<128, false><<<max_rows, kRopeThreads, 0, stream>>>(g.Hq, g.Hkv, c, n_active, pos_id, q, k_new, none);
     else
-        rope_kernel<64><<<max_rows, kRopeThreads, 0, stream>>>(g.Hq, g.Hkv, c, n_active, pos_id, q, k_new);
+        rope_kernel<64, false><<<max_rows, kRopeThreads, 0, stream>>>(g.Hq, g.Hkv, c, n_active, pos_id, q, k_new, none);
+    HPD_CUDA_TRY(cudaGetLastError());
+    return HPD_OK;
+}
+
+int launch_rope_append(const hpd_geom& g, int max_rows, int n_slots, const int32_t* n_active, const int32_t* pos_id,
+                       const int32_t* suffix_off, const int32_t* suffix_len, __nv_bfloat16* q, __nv_bfloat16* k_new,
+                       const __nv_bfloat16* v_new, __nv_bfloat16* suffix_k, __nv_bfloat16* suffix_v, int32_t* dev_status,
+                       cudaStream_t stream)
+{
+    if (max_rows <= 0) return HPD_OK;
+    const double c = -2.0 * log2(static_cast<double>(g.rope_theta)) / static_cast<double>(g.D);
+    const AppendDst ad{g.suffix_cap, static_cast<int64_t>(n_slots) * g.suffix_cap, suffix_off, suffix_len, v_new,
+                       suffix_k, suffix_v, dev_status};
+    if (g.D == 128)
+        rope_kernel<128, true><<<max_rows, kRopeThreads, 0, stream>>>(g.Hq, g.Hkv, c, n_active, pos_id, q, k_new, ad);
+    else
+        rope_kernel<64, true><<<max_rows, kRopeThreads, 0, stream>>>(g.Hq, g.Hkv, c, n_active, pos_id, q, k_new, ad);
     HPD_CUDA_TRY(cudaGetLastError());
     return HPD_OK;
 }

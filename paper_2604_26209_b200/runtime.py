@@ -67,26 +67,35 @@ class DeviceBatch:
         B.hpd_kv_append(self.g, self.s.n_slots, self.s.n_slots, self.meta.n_active, self.meta.suffix_off,
                         self.meta.suffix_len, self.k_new, self.v_new, self.suffix_k, self.suffix_v, self.meta.dev_status)
 
+    def rope_append(self):
+        B.hpd_rope_append(self.g, self.s.n_slots, self.s.n_slots, self.meta.n_active, self.meta.pos_id,
+                          self.meta.suffix_off, self.meta.suffix_len, self.q, self.k_new, self.v_new, self.suffix_k,
+                          self.suffix_v, self.meta.dev_status)
+
     def attn(self, suffix_includes_new=True, lse=True):
         s = self.s
         B.hpd_attn_decode(self.g, s.n_docs, s.n_slots, s.n_slots, s.total_prefix, self.q, self.prefix_k, self.prefix_v,
                           self.suffix_k, self.suffix_v, self.doc_prefix_len, self.meta, suffix_includes_new, self.o,
                           self.lse if lse else None)
 
-    def step(self, with_meta=True):
+    def step(self, with_meta=True, fused=True):
+        """One decode step; ``fused`` rotates and appends in one launch (hpd_rope_append) instead of two."""
         if with_meta:
             self.build_meta()
-        self.rope()
-        self.kv_append()
+        if fused:
+            self.rope_append()
+        else:
+            self.rope()
+            self.kv_append()
         self.attn(True)
 
-    def capture_step(self, with_meta=True):
+    def capture_step(self, with_meta=True, fused=True):
         """The step's launches captured once in a CUDA graph (call step() at least once before: the first call sets
         kernel attributes and builds tensor maps).  replay() then runs the same kernels without a host call each."""
         g = torch.cuda.CUDAGraph()
         torch.cuda.synchronize()
         with torch.cuda.graph(g):
-            self.step(with_meta=with_meta)
+            self.step(with_meta=with_meta, fused=fused)
         return g
 
     # -- read-back --------------------------------------------------------------------------

@@ -162,6 +162,49 @@ def test_step_matches_oracle(rt, name):
     assert np.max(np.abs(lse_gpu - want.lse)) <= 2e-2
 
 
+@pytest.mark.parametrize("name", ["tiny", "main_p2", "ragged_gap", "ragged_d64_g2", "cap3", "paper_j6_n16_k30"])
+def test_fused_rope_append_equals_the_two_calls(rt, name):
+    """hpd_rope_append = hpd_rope then hpd_kv_append, bit for bit: rotated q and k, the whole branch cache, the status."""
+    s = STRUCTS[name]()
+    tb = synth.make_tensors(s)
+    db, tabs = _run_step(rt, s, tb)
+    n = tabs["n_active"]
+    act = tabs["active_slot"][:n]
+    db2 = rt.DeviceBatch(s, tb)
+    db2.build_meta()
+    db2.set_step_inputs(tb["q"][act], tb["k_new"][act], tb["v_new"][act])
+    db2.rope_append()
+    db2.attn(True)
+    torch.cuda.synchronize()
+    assert db2.status() == db.status() == 0
+    for a in ("q", "k_new", "suffix_k", "suffix_v", "o"):
+        assert np.array_equal(rt.bits_of(getattr(db2, a)), rt.bits_of(getattr(db, a))), a
+
+
+def test_fused_rope_append_full_slab(rt):
+    """A full slab: the fused call still rotates the row's q and k, writes nothing to the cache and raises the status bit."""
+    from paper_2604_26209_b200 import binding
+    s = synth.config_custom("ovf", Hq=4, Hkv=1, D=64, theta=10000.0, cap=4, prefix_lens=[16], branch_cnts=[3],
+                            depth_hi=1, seed=14)
+    s.slot_depth[:] = [0, 4, 2]
+    tb = synth.make_tensors(s)
+    out = []
+    for fused in (False, True):
+        db = rt.DeviceBatch(s, tb)
+        db.build_meta()
+        db.set_step_inputs(tb["q"], tb["k_new"], tb["v_new"])
+        if fused:
+            db.rope_append()
+        else:
+            db.rope(); db.kv_append()
+        torch.cuda.synchronize()
+        assert db.status() == binding.HPD_S_OVERFLOW
+        out.append([rt.bits_of(getattr(db, a)).copy() for a in ("q", "k_new", "suffix_k", "suffix_v")])
+    for a, b in zip(*out):
+        assert np.array_equal(a, b)
+    assert np.array_equal(out[1][2][4:8], tb["suffix_k"][4:8])
+
+
 def test_graph_replay_equals_direct_calls(rt):
     """The step captured in a CUDA graph launches the same kernels on the same buffers: same bits."""
     s = synth.config_main(n_prompts=2)
