@@ -1,6 +1,7 @@
 // hpd_build_meta: per-step int32 bookkeeping tables and the attention work list (device side).
 //
-// Three small kernels, all on the caller's stream, no host synchronisation:
+// On the caller's stream, no host synchronisation.  Steps with up to 4096 documents take one launch
+// (meta_fused_kernel); larger ones three:
 //   doc_scan_kernel   exclusive scans over documents (prefix tokens, slots)
 //   compact_kernel    stable compaction of live slots -> row tables, rows-per-document CSR
 //   plan_kernel       split-KV policy + work list for the attention kernel; -1 fill of table tails
@@ -160,25 +161,14 @@ __device__ __forceinline__ int chunks_of(int L, int cand) {
     return (L + S - 1) / S;
 }
 
-__global__ void __launch_bounds__(kPlanThreads)
-plan_kernel(int n_docs, int n_slots, int G, int Hkv, int n_sm,
-            const int32_t* __restrict__ doc_prefix_len, const int32_t* __restrict__ doc_active_start,
-            const int32_t* __restrict__ n_active,
-            int32_t* __restrict__ active_slot, int32_t* __restrict__ doc_id, int32_t* __restrict__ branch_start,
-            int32_t* __restrict__ pos_id, int32_t* __restrict__ suffix_off, int32_t* __restrict__ suffix_len,
-            WsHeader* __restrict__ hdr, WorkItem* __restrict__ work, DocSplit* __restrict__ split,
-            int work_cap, int part_cap)
+// The split-KV plan, run by ONE block of THREADS threads (doc_active_start must be complete and visible).
+template <int THREADS>
+__device__ __forceinline__ void plan_block(int n_docs, int G, int Hkv, int n_sm,
+                                           const int32_t* doc_prefix_len, const int32_t* doc_active_start,
+                                           WsHeader* __restrict__ hdr, WorkItem* __restrict__ work, DocSplit* __restrict__ split,
+                                           int work_cap, int part_cap)
 {
-    if (blockIdx.x > 0) {
-        // tail fill: entries past n_active read -1 in every per-row table
-        const int na = *n_active;
-        for (int i = na + (blockIdx.x - 1) * kPlanThreads + threadIdx.x; i < n_slots; i += (gridDim.x - 1) * kPlanThreads) {
-            active_slot[i] = -1; doc_id[i] = -1; branch_start[i] = -1;
-            pos_id[i] = -1; suffix_off[i] = -1; suffix_len[i] = -1;
-        }
-        return;
-    }
-
+    constexpr int kPlanThreads = THREADS;
     __shared__ int sm[kPlanThreads / 32 + 1];
     __shared__ long long red[kCand * 2];
     __shared__ int s_choice;
@@ -191,7 +181,7 @@ plan_kernel(int n_docs, int n_slots, int G, int Hkv, int n_sm,
 #pragma unroll
         for (int c = 0; c < kCand; ++c) { items[c] = 0; prow[c] = 0; }
         for (int d = threadIdx.x; d < n_docs; d += kPlanThreads) {
-            const int rows = doc_active_start[d + 1] - doc_active_start[d];
+            const int rows = __ldcg(doc_active_start + d + 1) - __ldcg(doc_active_start + d);
             if (rows <= 0) continue;
             const int mb = (rows + rows_per_block - 1) / rows_per_block;
             const int L = doc_prefix_len[d];
@@ -234,7 +224,7 @@ plan_kernel(int n_docs, int n_slots, int G, int Hkv, int n_sm,
         const int d = base + threadIdx.x;
         int rows = 0, L = 0, mb = 0, ch = 0;
         if (d < n_docs) {
-            rows = doc_active_start[d + 1] - doc_active_start[d];
+            rows = __ldcg(doc_active_start + d + 1) - __ldcg(doc_active_start + d);
             L = doc_prefix_len[d];
             if (rows > 0) {
                 mb = (rows + rows_per_block - 1) / rows_per_block;
@@ -285,6 +275,151 @@ plan_kernel(int n_docs, int n_slots, int G, int Hkv, int n_sm,
     }
 }
 
+__global__ void __launch_bounds__(kPlanThreads)
+plan_kernel(int n_docs, int n_slots, int G, int Hkv, int n_sm,
+            const int32_t* __restrict__ doc_prefix_len, const int32_t* __restrict__ doc_active_start,
+            const int32_t* __restrict__ n_active,
+            int32_t* __restrict__ active_slot, int32_t* __restrict__ doc_id, int32_t* __restrict__ branch_start,
+            int32_t* __restrict__ pos_id, int32_t* __restrict__ suffix_off, int32_t* __restrict__ suffix_len,
+            WsHeader* __restrict__ hdr, WorkItem* __restrict__ work, DocSplit* __restrict__ split,
+            int work_cap, int part_cap)
+{
+    if (blockIdx.x > 0) {
+        // tail fill: entries past n_active read -1 in every per-row table
+        const int na = *n_active;
+        for (int i = na + (blockIdx.x - 1) * kPlanThreads + threadIdx.x; i < n_slots; i += (gridDim.x - 1) * kPlanThreads) {
+            active_slot[i] = -1; doc_id[i] = -1; branch_start[i] = -1;
+            pos_id[i] = -1; suffix_off[i] = -1; suffix_len[i] = -1;
+        }
+        return;
+    }
+    plan_block<kPlanThreads>(n_docs, G, Hkv, n_sm, doc_prefix_len, doc_active_start, hdr, work, split, work_cap, part_cap);
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// All of the above in ONE launch, for steps with at most kFusedDocs documents (the usual case).  Every block of 256
+// slots repeats the two cheap global steps for itself -- the scans over documents (kept in shared memory) and the
+// count of live slots before it and in total -- so that it can place its live slots' rows, its dead slots' -1 entries
+// at the tail, and its documents' CSR entries without waiting for any other block.  The block that finishes last
+// (counted in the workspace header) sees every block's CSR entries and writes the split-KV plan.
+// ---------------------------------------------------------------------------------------------------------------
+constexpr int kFusedDocs = 4096;
+constexpr int kFusedThreads = 256;
+
+__device__ __forceinline__ int count_alive(const uint8_t* __restrict__ slot_alive, int begin, int end)
+{
+    // live slots in [begin, end), 16 bytes at a time where the address allows
+    int cnt = 0;
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(slot_alive + begin);
+    int head = static_cast<int>((16 - (addr & 15)) & 15);
+    if (head > end - begin) head = end - begin;
+    for (int i = begin + threadIdx.x; i < begin + head; i += blockDim.x) cnt += slot_alive[i] != 0;
+    const int n_vec = (end - begin - head) / 16;
+    const uint4* v = reinterpret_cast<const uint4*>(slot_alive + begin + head);
+    for (int i = threadIdx.x; i < n_vec; i += blockDim.x) {
+        const uint4 w = v[i];
+        cnt += __popc(__vcmpne4(w.x, 0u) & 0x01010101u) + __popc(__vcmpne4(w.y, 0u) & 0x01010101u) +
+               __popc(__vcmpne4(w.z, 0u) & 0x01010101u) + __popc(__vcmpne4(w.w, 0u) & 0x01010101u);
+    }
+    for (int i = begin + head + n_vec * 16 + threadIdx.x; i < end; i += blockDim.x) cnt += slot_alive[i] != 0;
+    return cnt;
+}
+
+__global__ void __launch_bounds__(kFusedThreads)
+meta_fused_kernel(int n_docs, int n_slots, int32_t suffix_cap, int32_t pos_gap, int G, int Hkv, int n_sm,
+                  const int32_t* __restrict__ doc_prefix_len, const int32_t* __restrict__ doc_branch_cnt,
+                  const int32_t* __restrict__ slot_depth, const uint8_t* __restrict__ slot_alive,
+                  int32_t* __restrict__ doc_kv_start, int32_t* __restrict__ doc_slot_start, int32_t* doc_active_start,
+                  int32_t* __restrict__ active_slot, int32_t* __restrict__ doc_id, int32_t* __restrict__ branch_start,
+                  int32_t* __restrict__ pos_id, int32_t* __restrict__ suffix_off, int32_t* __restrict__ suffix_len,
+                  int32_t* __restrict__ n_active, WsHeader* hdr, WorkItem* __restrict__ work, DocSplit* __restrict__ split,
+                  int work_cap, int part_cap)
+{
+    __shared__ int sm[kFusedThreads / 32 + 1];
+    __shared__ int s_slot_start[kFusedDocs + 1];
+    __shared__ int s_last;
+    const int first = blockIdx.x * kFusedThreads;
+
+    // ---- scans over documents: slot starts stay in shared memory, block 0 also publishes both scans ----
+    {
+        int run_kv = 0, run_sl = 0;
+        for (int base = 0; base < n_docs; base += kFusedThreads) {
+            const int d = base + threadIdx.x;
+            const int l = d < n_docs ? doc_prefix_len[d] : 0;
+            const int c = d < n_docs ? doc_branch_cnt[d] : 0;
+            int tot_l, tot_c;
+            const int el = block_excl_scan<kFusedThreads>(l, sm, tot_l);
+            const int ec = block_excl_scan<kFusedThreads>(c, sm, tot_c);
+            if (d < n_docs) {
+                s_slot_start[d] = run_sl + ec;
+                if (blockIdx.x == 0) { doc_kv_start[d] = run_kv + el; doc_slot_start[d] = run_sl + ec; }
+            }
+            run_kv += tot_l;
+            run_sl += tot_c;
+        }
+        if (threadIdx.x == 0) {
+            s_slot_start[n_docs] = run_sl;
+            if (blockIdx.x == 0) { doc_kv_start[n_docs] = run_kv; doc_slot_start[n_docs] = run_sl; }
+        }
+    }
+    // ---- live slots before this block and in total ----
+    int before, total;
+    {
+        int tot;
+        block_excl_scan<kFusedThreads>(count_alive(slot_alive, 0, min(first, n_slots)), sm, tot);
+        before = tot;
+        block_excl_scan<kFusedThreads>(count_alive(slot_alive, min(first, n_slots), n_slots), sm, tot);
+        total = before + tot;
+    }
+    const int s = first + threadIdx.x;
+    const int alive = (s < n_slots) && slot_alive[s] != 0;
+    int tot;
+    const int excl = before + block_excl_scan<kFusedThreads>(alive, sm, tot);
+
+    if (s < n_slots) {
+        int lo = 0, hi = n_docs;           // invariant: slot_start[lo] <= s < slot_start[hi]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (s_slot_start[mid] <= s) lo = mid; else hi = mid;
+        }
+        const int d = lo;
+        const int j = s - s_slot_start[d];
+        if (j == 0) {
+            // first slot of document d: rows before it; documents without slots just before d share the value
+            doc_active_start[d] = excl;
+            for (int e = d - 1; e >= 0 && s_slot_start[e + 1] == s_slot_start[e]; --e) doc_active_start[e] = excl;
+        }
+        if (alive) {
+            const int depth = slot_depth[s];
+            const int bs = doc_prefix_len[d] + j * pos_gap;
+            active_slot[excl] = s;
+            doc_id[excl] = d;
+            branch_start[excl] = bs;
+            pos_id[excl] = bs + depth;
+            suffix_off[excl] = s * suffix_cap;
+            suffix_len[excl] = depth;
+        } else {
+            const int t = total + (s - excl);            // the dead slots fill the tail of every row table with -1
+            active_slot[t] = -1; doc_id[t] = -1; branch_start[t] = -1;
+            pos_id[t] = -1; suffix_off[t] = -1; suffix_len[t] = -1;
+        }
+    }
+    if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) {
+        *n_active = total;
+        doc_active_start[n_docs] = total;
+        for (int e = n_docs - 1; e >= 0 && s_slot_start[e + 1] == s_slot_start[e]; --e) doc_active_start[e] = total;
+    }
+
+    // ---- the block that finishes last writes the plan ----
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(&hdr->finished, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    plan_block<kFusedThreads>(n_docs, G, Hkv, n_sm, doc_prefix_len, doc_active_start, hdr, work, split, work_cap, part_cap);
+}
+
 }  // namespace
 
 WsLayout ws_layout(const hpd_geom& g, int max_docs, int max_slots, int n_sm)
@@ -320,6 +455,18 @@ int launch_build_meta(const hpd_geom& g, int n_docs, int n_slots, const int32_t*
     WorkItem* work = reinterpret_cast<WorkItem*>(ws + lay.off_work);
     DocSplit* split = reinterpret_cast<DocSplit*>(ws + lay.off_split);
 
+    if (n_docs <= kFusedDocs) {
+        // the header's arrival counter must read 0 at launch: plan_block leaves it so (hdr->finished = 0) after every
+        // step, and the very first step on a workspace finds whatever the caller's allocation holds -- clear it
+        HPD_CUDA_TRY(cudaMemsetAsync(&hdr->finished, 0, sizeof(hdr->finished), stream));
+        const int blocks = n_slots > 0 ? (n_slots + kFusedThreads - 1) / kFusedThreads : 1;
+        meta_fused_kernel<<<blocks, kFusedThreads, 0, stream>>>(
+            n_docs, n_slots, g.suffix_cap, pos_gap, g.Hq / g.Hkv, g.Hkv, n_sm, doc_prefix_len, doc_branch_cnt, slot_depth,
+            slot_alive, doc_kv_start, doc_slot_start, doc_active_start, active_slot, doc_id, branch_start, pos_id,
+            suffix_off, suffix_len, n_active, hdr, work, split, lay.work_cap, lay.part_cap);
+        HPD_CUDA_TRY(cudaGetLastError());
+        return HPD_OK;
+    }
     doc_scan_kernel<<<1, kScanThreads, 0, stream>>>(n_docs, doc_prefix_len, doc_branch_cnt, doc_kv_start, doc_slot_start);
     const int cblocks = n_slots > 0 ? (n_slots + kCompactThreads - 1) / kCompactThreads : 1;
     compact_kernel<<<cblocks, kCompactThreads, 0, stream>>>(
