@@ -23,6 +23,8 @@ def lib():
         _lib.hpdo_decode_step.restype = C.c_int
         _lib.hpdo_build_meta.restype = C.c_int
         _lib.hpdo_alg2_value_position.restype = C.c_int32
+        _lib.hpdo_build_meta_skeleton.restype = C.c_int
+        _lib.hpdo_decode_step_posorder.restype = C.c_int
     return _lib
 
 
@@ -164,3 +166,54 @@ def kv_append(geom, meta: Meta, k_rot, v_new, suffix_k: np.ndarray, suffix_v: np
     lib().hpdo_kv_append(C.c_int(geom.Hkv), C.c_int(geom.D), C.c_int(n), C.c_int32(geom.suffix_cap),
                          _p(soff), _p(slen), _p(k_rot), _p(v_new), _p(suffix_k), _p(suffix_v), _p(ovf))
     return ovf
+
+
+# ------------------------------------------------------------------------------------------
+# position-order mode (Sec. 4.3.2, Fig. 3, Sec. 4.4)
+# ------------------------------------------------------------------------------------------
+def build_meta_skeleton(doc_prefix_len, doc_branch_cnt, slot_depth, slot_alive, slot_vis, suffix_cap: int, pos_gap: int):
+    """Tables of the position-order mode: ``(Meta, prefix_vis)``; ``slot_vis[s]`` = prefix tokens of the group up to and
+    including the slot's attribute key."""
+    L, cnt, dep, vis = _i32(doc_prefix_len), _i32(doc_branch_cnt), _i32(slot_depth), _i32(slot_vis)
+    alive = np.ascontiguousarray(slot_alive, dtype=np.uint8)
+    nd, ns = len(L), len(dep)
+    z = lambda n: np.full(n, -7, dtype=np.int32)
+    m = Meta(z(nd + 1), z(nd + 1), z(nd + 1), z(ns), z(ns), z(ns), z(ns), z(ns), z(ns), 0)
+    pv = z(ns)
+    na = np.zeros(1, dtype=np.int32)
+    rc = lib().hpdo_build_meta_skeleton(C.c_int(nd), C.c_int(ns), _p(L), _p(cnt), _p(dep), _p(alive), _p(vis),
+                                        C.c_int32(suffix_cap), C.c_int32(pos_gap),
+                                        _p(m.doc_kv_start), _p(m.doc_slot_start), _p(m.doc_active_start),
+                                        _p(m.active_slot), _p(m.doc_id), _p(m.branch_start), _p(m.pos_id),
+                                        _p(m.suffix_off), _p(m.suffix_len), _p(pv), _p(na))
+    if rc != 0:
+        raise ValueError("oracle build_meta_skeleton: inconsistent arguments")
+    m.n_active = int(na[0])
+    return m, pv
+
+
+def decode_step_posorder(geom, meta: Meta, doc_prefix_len, slot_depth, slot_alive, slot_vis, k_max: int,
+                         q, k_new, v_new, prefix_k, prefix_v, suffix_k, suffix_v, n_threads: int = 0):
+    """One decode step under the position-order mask.  ``q, k_new, v_new`` per ACTIVE ROW (fp32).
+    Returns (StepOut, positions of the rows' new tokens)."""
+    n = meta.n_active
+    q, k_new, v_new = _f32(q), _f32(k_new), _f32(v_new)
+    assert q.shape == (n, geom.Hq, geom.D) and k_new.shape == (n, geom.Hkv, geom.D)
+    prefix_k, prefix_v, suffix_k, suffix_v = _f32(prefix_k), _f32(prefix_v), _f32(suffix_k), _f32(suffix_v)
+    L, dep, vis = _i32(doc_prefix_len), _i32(slot_depth), _i32(slot_vis)
+    alive = np.ascontiguousarray(slot_alive, dtype=np.uint8)
+    act, did = _i32(meta.active_slot[:n]), _i32(meta.doc_id[:n])
+    o = np.empty((n, geom.Hq, geom.D), dtype=np.float32)
+    lse = np.empty((n, geom.Hq), dtype=np.float32)
+    q_rot = np.empty((n, geom.Hq, geom.D), dtype=np.float32)
+    k_rot = np.empty((n, geom.Hkv, geom.D), dtype=np.float32)
+    pos = np.empty(max(n, 1), dtype=np.int32)
+    used = lib().hpdo_decode_step_posorder(
+        C.c_int(geom.Hq), C.c_int(geom.Hkv), C.c_int(geom.D), C.c_double(geom.rope_theta), C.c_double(geom.sm_scale),
+        _p(L), _p(meta.doc_kv_start), _p(meta.doc_slot_start), _p(dep), _p(alive), _p(vis),
+        C.c_int32(geom.suffix_cap), C.c_int32(k_max), C.c_int(n), _p(act), _p(did),
+        _p(q), _p(k_new), _p(v_new), _p(prefix_k), _p(prefix_v), _p(suffix_k), _p(suffix_v),
+        _p(o), _p(lse), _p(q_rot), _p(k_rot), _p(pos), C.c_int(n_threads))
+    if used < 0:
+        raise MemoryError("oracle decode_step_posorder: allocation failed")
+    return StepOut(o, lse, q_rot, k_rot, used), pos[:n]

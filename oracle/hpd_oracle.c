@@ -14,6 +14,9 @@
  *                                                        positional embeddings"), Sec. 4.4
  *   - per-branch attention                               Eq. 5-6: a value token depends on the
  *                                                        prompt and on its own earlier tokens only
+ *   - position-order attention (second mode)             Sec. 4.3.2 / Fig. 3 / Sec. 4.4: the mask the
+ *                                                        paper runs, causal in position-ID order over
+ *                                                        the whole stacked prompt, with K_max gaps
  *
  * Precision: inputs are fp32 values (the harness widens bf16 exactly); every product,
  * sum, exponential and trigonometric value is taken in fp64.  There is no blocking,
@@ -24,7 +27,9 @@
  * paper prints for its K_max = 7 figure; rope against closed forms and the relative-
  * position identity; attention against a full-matrix masked softmax in numpy, against
  * the library's causal SDPA, and against closed forms; the step against branch/document
- * permutation invariance.  Nothing in the paper prints an attention output value, so
+ * permutation invariance; the position-order mode against ordinary causal attention on the
+ * position-sorted sequence, against the fine-tuning mask of Sec. 4.4 written out in token
+ * order, and against the branch-local mode for single-branch groups.  Nothing in the paper prints an attention output value, so
  * beyond those pins the numeric values themselves are parity unpinned.
  */
 #include <math.h>
@@ -270,4 +275,168 @@ void hpdo_kv_append(int Hkv, int D, int n_active, int32_t suffix_cap,
         memcpy(suffix_k + dst, k_rot + (size_t)r * kvw, kvw * sizeof(float));
         memcpy(suffix_v + dst, v_new + (size_t)r * kvw, kvw * sizeof(float));
     }
+}
+
+
+/* ====================================================================================
+ * Position-order mode: the mask the paper's implementation runs (Sec. 4.3.2 "the triangular
+ * attention mask is computed using the position ID ordering"; Fig. 3 (a); Sec. 4.4).
+ *
+ * A group (one stacked prompt) is the model input s = cat(p, a_1..a_N): L tokens in memory, the
+ * last ones being the attribute-key tokens of the skeleton, attribute j ending at memory index
+ * vis[j] - 1.  Algorithm 2 leaves a gap of K_max position IDs after every attribute; with
+ * start(a_j) = end(a_{j-1}) + 1 (structure tokens are ignored, Sec. 4.3.1) this gives
+ *     position of prefix token t        = t + K_max * #{ j : vis[j] <= t }
+ *     position of value token k of j    = vis[j] + j*K_max + k        (= pos_id[end(a_j)] + k + 1)
+ * Value tokens are appended to the cache out of order; a new token sees every token of its group
+ * -- prompt, skeleton, cached value tokens of ANY branch, this step's new tokens -- whose position
+ * ID is not larger than its own.
+ * ==================================================================================== */
+
+/* Bookkeeping of the position-order mode: the tables of hpdo_build_meta with a per-slot anchor.
+ * slot_vis[s] = number of the group's prefix tokens up to and including the slot's attribute key;
+ * branch_start = slot_vis + j*pos_gap, prefix_vis[r] = slot_vis of the row's slot. */
+int hpdo_build_meta_skeleton(int n_docs, int n_slots,
+                             const int32_t* doc_prefix_len, const int32_t* doc_branch_cnt,
+                             const int32_t* slot_depth, const uint8_t* slot_alive, const int32_t* slot_vis,
+                             int32_t suffix_cap, int32_t pos_gap,
+                             int32_t* doc_kv_start, int32_t* doc_slot_start, int32_t* doc_active_start,
+                             int32_t* active_slot, int32_t* doc_id, int32_t* branch_start, int32_t* pos_id,
+                             int32_t* suffix_off, int32_t* suffix_len, int32_t* prefix_vis, int32_t* n_active)
+{
+    int kv = 0, sl = 0;
+    for (int d = 0; d < n_docs; ++d) {
+        doc_kv_start[d] = kv;   kv += doc_prefix_len[d];
+        doc_slot_start[d] = sl; sl += doc_branch_cnt[d];
+    }
+    doc_kv_start[n_docs] = kv;
+    doc_slot_start[n_docs] = sl;
+    if (sl != n_slots) return -1;
+    int r = 0;
+    for (int d = 0; d < n_docs; ++d) {
+        doc_active_start[d] = r;
+        for (int j = 0; j < doc_branch_cnt[d]; ++j) {
+            int s = doc_slot_start[d] + j;
+            if (slot_vis[s] < 0 || slot_vis[s] > doc_prefix_len[d]) return -1;
+            if (!slot_alive[s]) continue;
+            active_slot[r]  = s;
+            doc_id[r]       = d;
+            branch_start[r] = slot_vis[s] + j * pos_gap;
+            pos_id[r]       = branch_start[r] + slot_depth[s];
+            suffix_off[r]   = s * suffix_cap;
+            suffix_len[r]   = slot_depth[s];
+            prefix_vis[r]   = slot_vis[s];
+            ++r;
+        }
+    }
+    doc_active_start[n_docs] = r;
+    *n_active = r;
+    for (int i = r; i < n_slots; ++i)
+        active_slot[i] = doc_id[i] = branch_start[i] = pos_id[i] = suffix_off[i] = suffix_len[i] = prefix_vis[i] = -1;
+    return 0;
+}
+
+/* One decode step in position-order mode.  For every live row the visible tokens of its group are
+ * collected by comparing position IDs, one token at a time, and ordinary attention is taken over
+ * them (the query's own token last).  Inputs as hpdo_decode_step plus the slot tables; k_max is
+ * the position gap.  Returns the number of threads used, or -1. */
+int hpdo_decode_step_posorder(int Hq, int Hkv, int D, double theta, double scale,
+                              const int32_t* doc_prefix_len, const int32_t* doc_kv_start, const int32_t* doc_slot_start,
+                              const int32_t* slot_depth, const uint8_t* slot_alive, const int32_t* slot_vis,
+                              int32_t suffix_cap, int32_t k_max,
+                              int n_active, const int32_t* active_slot, const int32_t* doc_id,
+                              const float* q, const float* k_new, const float* v_new,
+                              const float* prefix_k, const float* prefix_v,
+                              const float* suffix_k, const float* suffix_v,
+                              float* o, float* lse, float* q_rot, float* k_rot, int32_t* pos_out,
+                              int n_threads)
+{
+    int used = 1, fail = 0;
+    size_t kvw = (size_t)Hkv * D, qw = (size_t)Hq * D;
+    /* position of every row's new token, and all rotated new keys (other rows may see them) */
+    int32_t* pos = (int32_t*)malloc(sizeof(int32_t) * (size_t)(n_active > 0 ? n_active : 1));
+    double* kr = (double*)malloc(sizeof(double) * kvw * (size_t)(n_active > 0 ? n_active : 1));
+    if (!pos || !kr) { free(pos); free(kr); return -1; }
+    for (int r = 0; r < n_active; ++r) {
+        int s = active_slot[r], d = doc_id[r];
+        int j = s - doc_slot_start[d];
+        pos[r] = slot_vis[s] + j * k_max + slot_depth[s];
+        hpdo_rope(Hkv, D, theta, pos[r], k_new + (size_t)r * kvw, kr + (size_t)r * kvw);
+        if (pos_out) pos_out[r] = pos[r];
+        if (k_rot) for (size_t i = 0; i < kvw; ++i) k_rot[(size_t)r * kvw + i] = (float)kr[(size_t)r * kvw + i];
+    }
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#endif
+#pragma omp parallel
+    {
+#ifdef _OPENMP
+#pragma omp single
+        used = omp_get_num_threads();
+#endif
+#pragma omp for schedule(dynamic, 1)
+        for (int r = 0; r < n_active; ++r) {
+            int d = doc_id[r], L = doc_prefix_len[d];
+            int s0 = doc_slot_start[d], s1 = doc_slot_start[d + 1];
+            int P = pos[r];
+            /* upper bound of visible tokens: the prefix, every cached token and every new token of the group */
+            size_t cap_n = (size_t)L + 1;
+            for (int s = s0; s < s1; ++s) cap_n += (size_t)slot_depth[s] + 1;
+            double* Kc = (double*)malloc(sizeof(double) * cap_n * kvw);
+            double* Vc = (double*)malloc(sizeof(double) * cap_n * kvw);
+            double* qr = (double*)malloc(sizeof(double) * qw);
+            double* orow = (double*)malloc(sizeof(double) * qw);
+            double* lrow = (double*)malloc(sizeof(double) * (size_t)Hq);
+            double* sc = (double*)malloc(sizeof(double) * cap_n);
+            if (!Kc || !Vc || !qr || !orow || !lrow || !sc) {
+                fail = 1;
+            } else {
+                size_t n = 0;
+                /* prompt and skeleton tokens, in memory order, by their Algorithm 2 position */
+                for (int t = 0; t < L; ++t) {
+                    int before = 0;
+                    for (int s = s0; s < s1; ++s) if (slot_vis[s] <= t) ++before;
+                    int pt = t + k_max * before;
+                    if (pt > P) continue;
+                    const float* pk = prefix_k + ((size_t)doc_kv_start[d] + t) * kvw;
+                    const float* pv = prefix_v + ((size_t)doc_kv_start[d] + t) * kvw;
+                    for (size_t i = 0; i < kvw; ++i) { Kc[n * kvw + i] = pk[i]; Vc[n * kvw + i] = pv[i]; }
+                    ++n;
+                }
+                /* cached value tokens of every branch of the group, alive or retired */
+                for (int s = s0; s < s1; ++s) {
+                    int j = s - s0;
+                    for (int k = 0; k < slot_depth[s]; ++k) {
+                        int pt = slot_vis[s] + j * k_max + k;
+                        if (pt > P) continue;
+                        const float* sk = suffix_k + ((size_t)s * suffix_cap + k) * kvw;
+                        const float* sv = suffix_v + ((size_t)s * suffix_cap + k) * kvw;
+                        for (size_t i = 0; i < kvw; ++i) { Kc[n * kvw + i] = sk[i]; Vc[n * kvw + i] = sv[i]; }
+                        ++n;
+                    }
+                }
+                /* this step's new tokens of the other live branches, then the row's own token last */
+                for (int pass = 0; pass < 2; ++pass) {
+                    for (int r2 = 0; r2 < n_active; ++r2) {
+                        if (doc_id[r2] != d) continue;
+                        if ((pass == 0) == (r2 == r)) continue;
+                        if (pos[r2] > P) continue;
+                        for (size_t i = 0; i < kvw; ++i) {
+                            Kc[n * kvw + i] = kr[(size_t)r2 * kvw + i];
+                            Vc[n * kvw + i] = v_new[(size_t)r2 * kvw + i];
+                        }
+                        ++n;
+                    }
+                }
+                hpdo_rope(Hq, D, theta, P, q + (size_t)r * qw, qr);
+                hpdo_causal_attention_row((int)n - 1, Hq, Hkv, D, scale, qr, Kc, Vc, orow, lrow, sc);
+                for (size_t i = 0; i < qw; ++i) o[(size_t)r * qw + i] = (float)orow[i];
+                if (lse) for (int h = 0; h < Hq; ++h) lse[(size_t)r * Hq + h] = (float)lrow[h];
+                if (q_rot) for (size_t i = 0; i < qw; ++i) q_rot[(size_t)r * qw + i] = (float)qr[i];
+            }
+            free(Kc); free(Vc); free(qr); free(orow); free(lrow); free(sc);
+        }
+    }
+    free(pos); free(kr);
+    return fail ? -1 : used;
 }

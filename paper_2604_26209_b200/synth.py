@@ -86,6 +86,8 @@ class Structure:
     docs_per_prompt: int = 1
     seed: int = 0
     eos_len: Optional[np.ndarray] = None  # int32 [n_slots], decode-loop workloads only
+    slot_vis: Optional[np.ndarray] = None  # int32 [n_slots], position-order workloads: prefix tokens of the group up to
+                                           # and including the slot's attribute key (the skeleton of Sec. 4.3.1)
 
     @property
     def n_docs(self) -> int:
@@ -164,6 +166,28 @@ def config_custom(name, Hq, Hkv, D, theta, cap, prefix_lens, branch_cnts, depth_
     depth = rng.integers(0, max(1, depth_hi), size=n_slots, dtype=np.int32) if n_slots else np.zeros(0, np.int32)
     alive = (rng.random(n_slots) < alive_frac).astype(np.uint8)
     return Structure(name, g, L, cnt, depth, alive, pos_gap, 1, int(L.shape[0]), seed)
+
+
+def config_skeleton(name, Hq, Hkv, D, theta, k_max, prompt_lens, branch_cnts, key_len_hi=4, depth_hi=None, seed=0,
+                    alive_frac=1.0) -> Structure:
+    """Position-order workload: every group is one stacked prompt, its prefix = ``prompt_lens[d]`` prompt tokens followed
+    by the skeleton, i.e. for each of its ``branch_cnts[d]`` branches an attribute key of 1..key_len_hi tokens (Sec.
+    4.3.1).  ``slot_vis`` marks where each branch's key ends; slab size and position gap are both ``k_max``."""
+    g = Geom(Hq=Hq, Hkv=Hkv, D=D, rope_theta=float(theta), sm_scale=float(1.0 / np.sqrt(D)), suffix_cap=k_max)
+    rng = np.random.default_rng(seed)
+    cnt = np.asarray(branch_cnts, dtype=np.int32)
+    n_slots = int(cnt.sum())
+    key_len = rng.integers(1, key_len_hi + 1, size=n_slots, dtype=np.int32)
+    L, vis, at = [], np.zeros(n_slots, np.int32), 0
+    for d, c in enumerate(cnt):
+        end = int(prompt_lens[d]) + np.cumsum(key_len[at:at + c])
+        vis[at:at + c] = end
+        L.append(int(end[-1]) if c else int(prompt_lens[d]))
+        at += c
+    depth_hi = k_max if depth_hi is None else depth_hi
+    depth = rng.integers(0, max(1, depth_hi), size=n_slots, dtype=np.int32)
+    alive = (rng.random(n_slots) < alive_frac).astype(np.uint8)
+    return Structure(name, g, np.asarray(L, dtype=np.int32), cnt, depth, alive, k_max, 1, len(cnt), seed, None, vis)
 
 
 def loop_step_state(s: Structure, step: int) -> Structure:
