@@ -42,6 +42,8 @@ def workload_prompts(workload: str) -> int:
         return 32
     if workload.startswith("main_p"):
         return int(workload[6:])
+    if workload.startswith("posorder_p"):
+        return int(workload[10:])
     raise SystemExit(f"unknown workload {workload}")
 
 
@@ -55,9 +57,20 @@ def rank_structure(workload: str, world: int, rank: int):
     mine = synth.shard_prompts(per_gpu * world, world, rank)
     if workload == "long":
         s = synth.config_long(n_prompts=len(mine), seed=mine.start)
+    elif workload.startswith("posorder_p"):
+        # the mask the paper runs (Sec. 4.3.2): every prompt is ONE group -- 4 stacked documents of 512 tokens as the
+        # prompt, then the skeleton of its 96 attribute keys -- shared by all of its 96 branches; K_max = 16
+        s = _posorder_structure(len(mine), mine.start)
+        s.n_prompts, s.docs_per_prompt = len(mine), 4
     else:
         s = synth.config_main(n_prompts=len(mine), seed=mine.start)
     return s, mine
+
+
+def _posorder_structure(n_prompts: int, seed: int):
+    g = synth.LLAMA3_8B
+    return synth.config_skeleton(f"posorder_p{n_prompts}", g["Hq"], g["Hkv"], g["D"], g["rope_theta"], 16,
+                                 [2048] * n_prompts, [96] * n_prompts, key_len_hi=4, seed=seed)
 
 
 def algorithmic_bytes(s) -> dict:
@@ -69,11 +82,25 @@ def algorithmic_bytes(s) -> dict:
     docs_live = np.unique(s.slot_doc()[alive])
     prefix = int(s.doc_prefix_len[docs_live].astype(np.int64).sum()) * row
     suffix = int((s.slot_depth[alive].astype(np.int64) + 1).sum()) * row
+    if s.slot_vis is not None:
+        # position-order mode: a group's cached tokens -- of retired slots too -- are read once for the rows behind them
+        sd = s.slot_doc()
+        last_live = np.full(s.n_docs, -1, np.int64)
+        np.maximum.at(last_live, sd[alive], np.nonzero(alive)[0])
+        seen = np.arange(s.n_slots) <= last_live[sd]
+        suffix = int((s.slot_depth[seen].astype(np.int64) + alive[seen]).sum()) * row
     n = int(alive.sum())
     qo = n * g.Hq * g.D * 2 * 2
     rope = 2 * n * (g.Hq + g.Hkv) * g.D * 2
     append = 2 * 2 * n * g.Hkv * g.D * 2
     keys = int((s.doc_prefix_len[s.slot_doc()[alive]].astype(np.int64) + s.slot_depth[alive] + 1).sum())
+    if s.slot_vis is not None:
+        # keys a row sees: the prefix up to its attribute key, every cached token of the group's slots up to its own
+        tok = s.slot_depth.astype(np.int64) + alive
+        cum = np.cumsum(tok)
+        first = np.concatenate([[0], np.cumsum(s.doc_branch_cnt)])[s.slot_doc()]
+        before_group = np.where(first > 0, cum[np.maximum(first - 1, 0)], 0)
+        keys = int((s.slot_vis.astype(np.int64) + cum - before_group)[alive].sum())
     return dict(attn=prefix + suffix + qo, prefix=prefix, suffix=suffix, qo=qo, rope=rope, append=append,
                 flops=4 * g.D * g.Hq * keys, n_active=n)
 
@@ -353,7 +380,7 @@ def run_ours(args):
                    "sample": f"{rows_done} rows ({args.cpu_rows} evenly spaced rows of the {n}-row step per pass), "
                              f"{t_cpu:.1f} s of oracle time"}
         comparison = None
-        if world == 1 and not args.no_comparison:
+        if world == 1 and not args.no_comparison and s.slot_vis is None:
             # the in-repo comparison: every branch with a private physical copy of [prefix ; branch tokens]
             free_b, _ = torch.cuda.mem_get_info()
             row_b = s.geom.Hkv * s.geom.D * 2 * 2
@@ -392,7 +419,8 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
             "ms_per_step": ms_head / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": s.name, "prompts_per_gpu": s.n_prompts, "global_prompts": s.n_prompts * world,
+            "config": {"workload": s.name, "mask": "position order (Sec. 4.3.2)" if s.slot_vis is not None else "branch-local (Eq. 5-6)",
+                       "prompts_per_gpu": s.n_prompts, "global_prompts": s.n_prompts * world,
                        "branches_per_prompt": 96, "docs_per_prompt": s.docs_per_prompt, "n_active_per_gpu": n,
                        "geometry": "Hq32/Hkv8/D128", "layers": 1,
                        "l2": f"inputs larger than L2 ({ab['attn'] / 1e6:.0f} MB touched per step vs 126 MB L2); no flush",

@@ -158,6 +158,48 @@ int hpd_attn_decode(const hpd_geom* geom /*host*/, int n_docs, int max_rows, int
                     void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream);
 
 /*
+ * Position-order mode: the mask the paper's implementation runs (Sec. 4.3.2: "the triangular attention
+ * mask is computed using the position ID ordering"; Fig. 3; Sec. 4.4; Algorithm 2).  A "document" of the
+ * tables is then a whole stacked prompt: its prefix is the prompt followed by the skeleton, i.e. the
+ * attribute-key tokens of its slots in slot order, and Algorithm 2 leaves a gap of pos_gap = K_max
+ * position IDs behind every attribute key.  A new token sees every token of its group whose position ID
+ * is not larger than its own: the prefix up to and including its own attribute key, and the cached
+ * tokens of every slot of the group up to and including its own -- retired slots too, their tokens stay
+ * in the cache (Sec. 4.3.4) -- which in the lock-step loop of Algorithm 1 is exactly the pattern of the
+ * fine-tuning mask of Sec. 4.4.
+ *
+ * hpd_build_meta_skeleton -- hpd_build_meta with a per-slot anchor:
+ *   slot_vis[n_slots] (dev)   prefix tokens of the slot's group up to and including its attribute key
+ *                             (= end(a_j) + 1 in Algorithm 2's notation; 0 <= slot_vis <= L_d, ascending
+ *                             inside a group)
+ *   branch_start[r] = slot_vis + j*pos_gap   (= pos_id[end(a_j)] + 1 of Algorithm 2)
+ *   prefix_vis[r]   = slot_vis of the row's slot (n_slots entries, -1 past n_active)
+ * Everything else as hpd_build_meta.
+ *
+ * hpd_attn_decode_posorder -- the attention under that mask.  Arguments as hpd_attn_decode, with the
+ * slot tables (doc_slot_start, active_slot from the builder; the caller's slot_depth and slot_alive) in
+ * place of suffix_off / suffix_len, and prefix_vis.  A slot's slab starts at row slot*suffix_cap; it
+ * holds slot_depth tokens, one more for live slots when suffix_includes_new is set.  A group may have at
+ * most 128 slots (larger groups set HPD_S_BAD_TABLE and their rows see the prefix only).
+ */
+int hpd_build_meta_skeleton(const hpd_geom* geom /*host*/, int n_docs, int n_slots,
+                            const int32_t* doc_prefix_len, const int32_t* doc_branch_cnt,
+                            const int32_t* slot_depth, const uint8_t* slot_alive, const int32_t* slot_vis, int32_t pos_gap,
+                            int32_t* doc_kv_start, int32_t* doc_slot_start, int32_t* doc_active_start,
+                            int32_t* active_slot, int32_t* doc_id, int32_t* branch_start, int32_t* pos_id,
+                            int32_t* suffix_off, int32_t* suffix_len, int32_t* prefix_vis, int32_t* n_active,
+                            void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream);
+int hpd_attn_decode_posorder(const hpd_geom* geom /*host*/, int n_docs, int max_rows, int n_slots, int total_prefix_tokens,
+                             const void* q, const void* prefix_k, const void* prefix_v,
+                             const void* suffix_k, const void* suffix_v,
+                             const int32_t* doc_kv_start, const int32_t* doc_prefix_len, const int32_t* doc_active_start,
+                             const int32_t* doc_slot_start, const int32_t* doc_id, const int32_t* active_slot,
+                             const int32_t* slot_depth, const uint8_t* slot_alive, const int32_t* prefix_vis,
+                             const int32_t* n_active, int suffix_includes_new,
+                             void* o, float* lse,
+                             void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream);
+
+/*
  * std_attn_decode -- the in-repo comparison: standard batched decode in which every branch is a
  * sequence of its own with a private physical copy of [prefix ; branch tokens] (parallel streams
  * as batch elements, Sec. 2; standard batched inference, Sec. 4.3.6).  Same math as

@@ -18,7 +18,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libhpd.so")
 
 EXPORTS = ("hpd_strerror", "hpd_last_cuda_error", "hpd_workspace_bytes", "hpd_build_meta", "hpd_rope",
-           "hpd_kv_append", "hpd_rope_append", "hpd_attn_decode", "std_workspace_bytes", "std_attn_decode",
+           "hpd_kv_append", "hpd_rope_append", "hpd_attn_decode", "hpd_build_meta_skeleton", "hpd_attn_decode_posorder", "std_workspace_bytes", "std_attn_decode",
            "std_attn_decode_static_max_bytes", "std_attn_decode_static")
 
 HPD_S_OVERFLOW, HPD_S_BAD_TABLE, HPD_S_TIMEOUT = 1, 2, 4
@@ -54,6 +54,12 @@ def load() -> C.CDLL:
         lib.hpd_build_meta.restype = C.c_int
         lib.hpd_build_meta.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int, vp, vp, vp, vp, C.c_int32] + [vp] * 10 + \
                                       [vp, C.c_size_t, vp, vp]
+        lib.hpd_build_meta_skeleton.restype = C.c_int
+        lib.hpd_build_meta_skeleton.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int, vp, vp, vp, vp, vp, C.c_int32] + \
+                                               [vp] * 11 + [vp, C.c_size_t, vp, vp]
+        lib.hpd_attn_decode_posorder.restype = C.c_int
+        lib.hpd_attn_decode_posorder.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int, C.c_int, C.c_int] + [vp] * 15 + \
+                                                [C.c_int, vp, vp, vp, C.c_size_t, vp, vp]
         lib.hpd_rope.restype = C.c_int
         lib.hpd_rope.argtypes = [C.POINTER(HpdGeom), C.c_int, vp, vp, vp, vp, vp]
         lib.hpd_kv_append.restype = C.c_int
@@ -122,6 +128,7 @@ class MetaTables:
     n_active: torch.Tensor
     workspace: torch.Tensor
     dev_status: torch.Tensor
+    prefix_vis: Optional[torch.Tensor] = None      # position-order mode only
 
     NAMES = ("doc_kv_start", "doc_slot_start", "doc_active_start", "active_slot", "doc_id", "branch_start",
              "pos_id", "suffix_off", "suffix_len")
@@ -132,7 +139,7 @@ class MetaTables:
         ws = torch.empty(max(hpd_workspace_bytes(geom, n_docs, n_slots, total_prefix), 256), dtype=torch.uint8, device=device)
         return MetaTables(i32(n_docs + 1), i32(n_docs + 1), i32(n_docs + 1), *[i32(n_slots) for _ in range(6)],
                           torch.zeros(1, dtype=torch.int32, device=device), ws,
-                          torch.zeros(1, dtype=torch.int32, device=device))
+                          torch.zeros(1, dtype=torch.int32, device=device), i32(n_slots))
 
 
 def hpd_build_meta(geom, n_docs, n_slots, doc_prefix_len, doc_branch_cnt, slot_depth, slot_alive, pos_gap, m: MetaTables):
@@ -143,6 +150,30 @@ def hpd_build_meta(geom, n_docs, n_slots, doc_prefix_len, doc_branch_cnt, slot_d
                                _ptr(m.pos_id), _ptr(m.suffix_off), _ptr(m.suffix_len), _ptr(m.n_active),
                                _ptr(m.workspace), m.workspace.numel(), _ptr(m.dev_status), _stream())
     _check(rc, "hpd_build_meta")
+
+
+def hpd_build_meta_skeleton(geom, n_docs, n_slots, doc_prefix_len, doc_branch_cnt, slot_depth, slot_alive, slot_vis, pos_gap,
+                            m: MetaTables):
+    g = make_geom(geom)
+    rc = load().hpd_build_meta_skeleton(C.byref(g), n_docs, n_slots, _ptr(doc_prefix_len), _ptr(doc_branch_cnt),
+                                        _ptr(slot_depth), _ptr(slot_alive), _ptr(slot_vis), int(pos_gap),
+                                        _ptr(m.doc_kv_start), _ptr(m.doc_slot_start), _ptr(m.doc_active_start),
+                                        _ptr(m.active_slot), _ptr(m.doc_id), _ptr(m.branch_start), _ptr(m.pos_id),
+                                        _ptr(m.suffix_off), _ptr(m.suffix_len), _ptr(m.prefix_vis), _ptr(m.n_active),
+                                        _ptr(m.workspace), m.workspace.numel(), _ptr(m.dev_status), _stream())
+    _check(rc, "hpd_build_meta_skeleton")
+
+
+def hpd_attn_decode_posorder(geom, n_docs, max_rows, n_slots, total_prefix_tokens, q, prefix_k, prefix_v, suffix_k, suffix_v,
+                             doc_prefix_len, slot_depth, slot_alive, m: MetaTables, suffix_includes_new, o, lse=None):
+    g = make_geom(geom)
+    rc = load().hpd_attn_decode_posorder(C.byref(g), n_docs, max_rows, n_slots, total_prefix_tokens, _ptr(q), _ptr(prefix_k),
+                                         _ptr(prefix_v), _ptr(suffix_k), _ptr(suffix_v), _ptr(m.doc_kv_start),
+                                         _ptr(doc_prefix_len), _ptr(m.doc_active_start), _ptr(m.doc_slot_start),
+                                         _ptr(m.doc_id), _ptr(m.active_slot), _ptr(slot_depth), _ptr(slot_alive),
+                                         _ptr(m.prefix_vis), _ptr(m.n_active), int(bool(suffix_includes_new)), _ptr(o),
+                                         _ptr(lse), _ptr(m.workspace), m.workspace.numel(), _ptr(m.dev_status), _stream())
+    _check(rc, "hpd_attn_decode_posorder")
 
 
 def hpd_rope(geom, max_rows, n_active, pos_id, q, k_new):

@@ -74,13 +74,13 @@ size_t hpd_workspace_bytes(const hpd_geom* geom, int max_docs, int max_slots, in
     return ws_layout(*geom, max_docs, max_slots, sm_count()).total;
 }
 
-int hpd_build_meta(const hpd_geom* geom, int n_docs, int n_slots,
-                   const int32_t* doc_prefix_len, const int32_t* doc_branch_cnt,
-                   const int32_t* slot_depth, const uint8_t* slot_alive, int32_t pos_gap,
-                   int32_t* doc_kv_start, int32_t* doc_slot_start, int32_t* doc_active_start,
-                   int32_t* active_slot, int32_t* doc_id, int32_t* branch_start, int32_t* pos_id,
-                   int32_t* suffix_off, int32_t* suffix_len, int32_t* n_active,
-                   void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream)
+static int build_meta_common(const hpd_geom* geom, int n_docs, int n_slots,
+                             const int32_t* doc_prefix_len, const int32_t* doc_branch_cnt,
+                             const int32_t* slot_depth, const uint8_t* slot_alive, const int32_t* slot_vis, int32_t pos_gap,
+                             int32_t* doc_kv_start, int32_t* doc_slot_start, int32_t* doc_active_start,
+                             int32_t* active_slot, int32_t* doc_id, int32_t* branch_start, int32_t* pos_id,
+                             int32_t* suffix_off, int32_t* suffix_len, int32_t* prefix_vis, int32_t* n_active,
+                             void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream)
 {
     int rc = geom_check(geom);
     if (rc != HPD_OK) return rc;
@@ -98,7 +98,34 @@ int hpd_build_meta(const hpd_geom* geom, int n_docs, int n_slots,
     return launch_build_meta(*geom, n_docs, n_slots, doc_prefix_len, doc_branch_cnt, slot_depth, slot_alive, pos_gap,
                              doc_kv_start, doc_slot_start, doc_active_start, active_slot, doc_id, branch_start, pos_id,
                              suffix_off, suffix_len, n_active, workspace, lay, n_sm, dev_status,
-                             static_cast<cudaStream_t>(stream));
+                             static_cast<cudaStream_t>(stream), slot_vis, prefix_vis);
+}
+
+int hpd_build_meta(const hpd_geom* geom, int n_docs, int n_slots,
+                   const int32_t* doc_prefix_len, const int32_t* doc_branch_cnt,
+                   const int32_t* slot_depth, const uint8_t* slot_alive, int32_t pos_gap,
+                   int32_t* doc_kv_start, int32_t* doc_slot_start, int32_t* doc_active_start,
+                   int32_t* active_slot, int32_t* doc_id, int32_t* branch_start, int32_t* pos_id,
+                   int32_t* suffix_off, int32_t* suffix_len, int32_t* n_active,
+                   void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream)
+{
+    return build_meta_common(geom, n_docs, n_slots, doc_prefix_len, doc_branch_cnt, slot_depth, slot_alive, nullptr, pos_gap,
+                             doc_kv_start, doc_slot_start, doc_active_start, active_slot, doc_id, branch_start, pos_id,
+                             suffix_off, suffix_len, nullptr, n_active, workspace, workspace_bytes, dev_status, stream);
+}
+
+int hpd_build_meta_skeleton(const hpd_geom* geom, int n_docs, int n_slots,
+                            const int32_t* doc_prefix_len, const int32_t* doc_branch_cnt,
+                            const int32_t* slot_depth, const uint8_t* slot_alive, const int32_t* slot_vis, int32_t pos_gap,
+                            int32_t* doc_kv_start, int32_t* doc_slot_start, int32_t* doc_active_start,
+                            int32_t* active_slot, int32_t* doc_id, int32_t* branch_start, int32_t* pos_id,
+                            int32_t* suffix_off, int32_t* suffix_len, int32_t* prefix_vis, int32_t* n_active,
+                            void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream)
+{
+    if (n_slots > 0 && (!slot_vis || !prefix_vis)) return HPD_E_ARG;
+    return build_meta_common(geom, n_docs, n_slots, doc_prefix_len, doc_branch_cnt, slot_depth, slot_alive, slot_vis, pos_gap,
+                             doc_kv_start, doc_slot_start, doc_active_start, active_slot, doc_id, branch_start, pos_id,
+                             suffix_off, suffix_len, prefix_vis, n_active, workspace, workspace_bytes, dev_status, stream);
 }
 
 int hpd_rope(const hpd_geom* geom, int max_rows, const int32_t* n_active, const int32_t* pos_id,
@@ -146,14 +173,19 @@ int hpd_rope_append(const hpd_geom* geom, int max_rows, int n_slots, const int32
                               static_cast<__nv_bfloat16*>(suffix_v), dev_status, static_cast<cudaStream_t>(stream));
 }
 
-int hpd_attn_decode(const hpd_geom* geom, int n_docs, int max_rows, int n_slots, int total_prefix_tokens,
-                    const void* q, const void* prefix_k, const void* prefix_v,
-                    const void* suffix_k, const void* suffix_v,
-                    const int32_t* doc_kv_start, const int32_t* doc_prefix_len, const int32_t* doc_active_start,
-                    const int32_t* doc_id, const int32_t* suffix_off, const int32_t* suffix_len,
-                    const int32_t* n_active, int suffix_includes_new,
-                    void* o, float* lse,
-                    void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream)
+struct OrderTables {                 // extra tables of the position-order mode (all null in the branch-local mode)
+    const int32_t *doc_slot_start, *active_slot, *slot_depth, *prefix_vis;
+    const uint8_t* slot_alive;
+};
+
+static int attn_common(const hpd_geom* geom, int n_docs, int max_rows, int n_slots, int total_prefix_tokens,
+                       const void* q, const void* prefix_k, const void* prefix_v,
+                       const void* suffix_k, const void* suffix_v,
+                       const int32_t* doc_kv_start, const int32_t* doc_prefix_len, const int32_t* doc_active_start,
+                       const int32_t* doc_id, const int32_t* suffix_off, const int32_t* suffix_len,
+                       const OrderTables& ord, const int32_t* n_active, int suffix_includes_new,
+                       void* o, float* lse,
+                       void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream)
 {
     int rc = geom_check(geom);
     if (rc != HPD_OK) return rc;
@@ -161,8 +193,11 @@ int hpd_attn_decode(const hpd_geom* geom, int n_docs, int max_rows, int n_slots,
     if (attn_packed_columns(*geom) > kMaxPackedColumns) return HPD_E_CAPACITY;
     if (n_docs < 0 || max_rows < 0 || n_slots < 0 || total_prefix_tokens < 0) return HPD_E_ARG;
     if (max_rows == 0 || n_docs == 0) return HPD_OK;
+    const bool order = ord.active_slot != nullptr;
     if (!q || !suffix_k || !suffix_v || !doc_kv_start || !doc_prefix_len || !doc_active_start || !doc_id ||
-        !suffix_off || !suffix_len || !n_active || !o || !workspace) return HPD_E_ARG;
+        !n_active || !o || !workspace) return HPD_E_ARG;
+    if (!order && (!suffix_off || !suffix_len)) return HPD_E_ARG;
+    if (order && (!ord.doc_slot_start || !ord.slot_depth || !ord.slot_alive || !ord.prefix_vis)) return HPD_E_ARG;
     if (total_prefix_tokens > 0 && (!prefix_k || !prefix_v)) return HPD_E_ARG;
     if (!aligned16(q) || !aligned16(prefix_k) || !aligned16(prefix_v) || !aligned16(suffix_k) ||
         !aligned16(suffix_v) || !aligned16(o) || !aligned16(workspace)) return HPD_E_ARG;
@@ -180,11 +215,44 @@ int hpd_attn_decode(const hpd_geom* geom, int n_docs, int max_rows, int n_slots,
     a.doc_kv_start = doc_kv_start; a.doc_prefix_len = doc_prefix_len; a.doc_active_start = doc_active_start;
     a.doc_id = doc_id; a.suffix_off = suffix_off; a.suffix_len = suffix_len; a.n_active = n_active;
     a.suffix_extra = suffix_includes_new ? 1 : 0;
+    a.doc_slot_start = ord.doc_slot_start; a.active_slot = ord.active_slot; a.slot_depth = ord.slot_depth;
+    a.prefix_vis = ord.prefix_vis; a.slot_alive = ord.slot_alive;
     a.o = static_cast<__nv_bfloat16*>(o);
     a.lse = lse;
     a.workspace = workspace; a.lay = lay; a.dev_status = dev_status;
     a.stream = static_cast<cudaStream_t>(stream);
     return launch_attn_tc(a);
+}
+
+int hpd_attn_decode(const hpd_geom* geom, int n_docs, int max_rows, int n_slots, int total_prefix_tokens,
+                    const void* q, const void* prefix_k, const void* prefix_v,
+                    const void* suffix_k, const void* suffix_v,
+                    const int32_t* doc_kv_start, const int32_t* doc_prefix_len, const int32_t* doc_active_start,
+                    const int32_t* doc_id, const int32_t* suffix_off, const int32_t* suffix_len,
+                    const int32_t* n_active, int suffix_includes_new,
+                    void* o, float* lse,
+                    void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream)
+{
+    return attn_common(geom, n_docs, max_rows, n_slots, total_prefix_tokens, q, prefix_k, prefix_v, suffix_k, suffix_v,
+                       doc_kv_start, doc_prefix_len, doc_active_start, doc_id, suffix_off, suffix_len, OrderTables{},
+                       n_active, suffix_includes_new, o, lse, workspace, workspace_bytes, dev_status, stream);
+}
+
+int hpd_attn_decode_posorder(const hpd_geom* geom, int n_docs, int max_rows, int n_slots, int total_prefix_tokens,
+                             const void* q, const void* prefix_k, const void* prefix_v,
+                             const void* suffix_k, const void* suffix_v,
+                             const int32_t* doc_kv_start, const int32_t* doc_prefix_len, const int32_t* doc_active_start,
+                             const int32_t* doc_slot_start, const int32_t* doc_id, const int32_t* active_slot,
+                             const int32_t* slot_depth, const uint8_t* slot_alive, const int32_t* prefix_vis,
+                             const int32_t* n_active, int suffix_includes_new,
+                             void* o, float* lse,
+                             void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream)
+{
+    if (max_rows > 0 && n_docs > 0 && !active_slot) return HPD_E_ARG;
+    const OrderTables ord{doc_slot_start, active_slot, slot_depth, prefix_vis, slot_alive};
+    return attn_common(geom, n_docs, max_rows, n_slots, total_prefix_tokens, q, prefix_k, prefix_v, suffix_k, suffix_v,
+                       doc_kv_start, doc_prefix_len, doc_active_start, doc_id, nullptr, nullptr, ord,
+                       n_active, suffix_includes_new, o, lse, workspace, workspace_bytes, dev_status, stream);
 }
 
 static int std_splits(const hpd_geom* g, int max_rows, int max_seq_len)

@@ -73,13 +73,13 @@ template <int D> struct Cfg {
     static constexpr int OFF_K = OFF_STAGE + 8 * 2048;
     static constexpr int OFF_V = OFF_K + 2 * NK * KV_BYTES;
     static constexpr int OFF_MISC = OFF_V + 2 * NV * KV_BYTES;
-    static constexpr int SMEM = OFF_MISC + 3072;                 // + misc; the dynamic segment itself is 1024-B aligned
+    static constexpr int SMEM = OFF_MISC + 4096;                 // + misc; the dynamic segment itself is 1024-B aligned
     static_assert(NK <= kMaxStages && NV <= kMaxStages, "barrier storage");
 };
 static_assert(Cfg<128>::SMEM <= 232448, "shared memory budget");
 
-struct SufMaps {                            // tensor maps of the branch cache, one per box height
-    CUtensorMap k[kBoxKinds];               // 4, 8, 12, 16 rows
+template <int NK> struct SufMapsT {        // tensor maps of the branch cache, one per box height
+    CUtensorMap k[NK];                      // NK = 4: 4, 8, 12, 16 rows (padded packing); NK = 16: 1 .. 16 rows (exact)
     CUtensorMap v[16];                      // 1 .. 16 rows
 };
 
@@ -110,8 +110,11 @@ struct UnitDesc {
     int pad[2];
     uint16_t cs[kM];     // per branch: packed column of its first cached token
     uint16_t len[kM];    // per branch: cached tokens visible (0 for a bad table entry)
+    // position-order mode: the branches above are ALL slots of the group up to the unit's last row (live or retired);
+    uint16_t ridx[kM];   // per row-branch of the unit: its index among them
+    int32_t pvis[kM];    // per row-branch: prefix tokens of this unit's chunk it may see
 };
-static_assert(sizeof(UnitDesc) == 48 + 4 * kM, "descriptor size");
+static_assert(sizeof(UnitDesc) == 48 + 10 * kM, "descriptor size");
 
 struct Misc {
     unsigned long long q_full[2], q_empty[2];
@@ -124,7 +127,7 @@ struct Misc {
     UnitDesc desc[2];    // one per pipeline
 };
 
-static_assert(sizeof(Misc) <= 3072, "misc block");
+static_assert(sizeof(Misc) <= 4096, "misc block");
 
 // ------------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -241,7 +244,7 @@ __device__ __forceinline__ Unit read_unit(const UnitDesc& d) {
 // 16 rows high and may read up to three rows past the branch's length (their columns are masked); V boxes (EXACT) have
 // the exact height, because whatever lies beyond a branch's length in the cache -- possibly NaN -- would otherwise be
 // multiplied by a zero probability.
-template <int D, bool EXACT>
+template <int D, bool EXACT, int PAD>
 __device__ __forceinline__ void fill_tile(const Unit& u, int t, const int (&cs)[kRounds], const int (&len)[kRounds], const int (&off)[kRounds],
                                           int lane, uint8_t* tile, unsigned long long* full, const CUtensorMap* pre, const CUtensorMap* suf)
 {
@@ -258,21 +261,21 @@ __device__ __forceinline__ void fill_tile(const Unit& u, int t, const int (&cs)[
         int rows_mine = 0;
 #pragma unroll
         for (int r = 0; r < kRounds; ++r) {
-            const int plen = EXACT ? len[r] : (len[r] + kPad - 1) & ~(kPad - 1);
+            const int plen = EXACT ? len[r] : (len[r] + PAD - 1) & ~(PAD - 1);
             rows_mine += max(0, min(cs[r] + plen, c_hi) - max(cs[r], c_lo));
         }
         const int rows_all = __reduce_add_sync(0xffffffffu, rows_mine);
         if (lane == 0) mbar_expect_tx(full, static_cast<uint32_t>(rows_all) * D * 2);
 #pragma unroll
         for (int r = 0; r < kRounds; ++r) {
-            const int plen = EXACT ? len[r] : (len[r] + kPad - 1) & ~(kPad - 1);
+            const int plen = EXACT ? len[r] : (len[r] + PAD - 1) & ~(PAD - 1);
             const int lo = max(cs[r], c_lo), hi = min(cs[r] + plen, c_hi);
             int n = hi - lo;
             int row = off[r] + (lo - cs[r]);
             int col = lo - c_lo;
             while (n > 0) {
                 const int hb = min(n, 16);
-                const CUtensorMap* m = EXACT ? &suf[hb - 1] : &suf[hb / 4 - 1];
+                const CUtensorMap* m = (EXACT || PAD == 1) ? &suf[hb - 1] : &suf[hb / 4 - 1];
                 for (int h = 0; h < C::HALVES; ++h)
                     tma_load_3d(tile + h * kKHalf + col * 128, m, full, h * 64, u.head, row);
                 row += hb; col += hb; n -= hb;
@@ -284,11 +287,19 @@ __device__ __forceinline__ void fill_tile(const Unit& u, int t, const int (&cs)[
 // ------------------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------------------
-template <int D>
+// ORDER = false: branch-local mask (Eq. 5-6): a row sees its document's prefix and its own branch's cached tokens.
+// ORDER = true:  position-order mask (Sec. 4.3.2, Fig. 3): a group is a whole stacked prompt; a row sees the first
+//                prefix_vis[row] prefix tokens (prompt and the skeleton up to its own attribute key) and the cached
+//                tokens of every slot of the group up to and including its own -- live or retired --, which is "position
+//                ID not larger than mine" under Algorithm 2's K_max gaps.  Branch tokens are then packed without padding
+//                (K boxes of the exact height), so a row's visible packed columns are one range starting at 0.
+template <int D, bool ORDER>
 __global__ void __launch_bounds__(kThreads, 1)
 hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                   const __grid_constant__ CUtensorMap map_v, const __grid_constant__ SufMaps smaps, const TcParams p)
+                   const __grid_constant__ CUtensorMap map_v, const __grid_constant__ SufMapsT<ORDER ? 16 : kBoxKinds> smaps,
+                   const TcParams p)
 {
+    constexpr int PAD = ORDER ? 1 : kPad;
     using C = Cfg<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
     Misc* misc = reinterpret_cast<Misc*>(smem + C::OFF_MISC);
@@ -364,20 +375,41 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         WorkItem it2 = item_of(w2), it1 = item_of(w1), it0 = item_of(w0);
         int das1 = p.a.doc_active_start[it1.doc], dks1 = p.a.doc_kv_start[it1.doc];
         int das0 = p.a.doc_active_start[it0.doc], dks0 = p.a.doc_kv_start[it0.doc];
-        int rl0[kRounds], ro0[kRounds];                                        // raw branch table of unit i
-        auto load_tab = [&](int w, const WorkItem& it, int das, int* rl, int* ro) {
+        // position-order mode: first slot of the group and of the next one
+        int dss1 = 0, dse1 = 0, dss0 = 0, dse0 = 0;
+        if constexpr (ORDER) {
+            dss1 = p.a.doc_slot_start[it1.doc]; dse1 = p.a.doc_slot_start[it1.doc + 1];
+            dss0 = p.a.doc_slot_start[it0.doc]; dse0 = p.a.doc_slot_start[it0.doc + 1];
+        }
+        // raw branch table of unit i.  Branch-local mode: per row, cached tokens (rl) and slab start (ro).  Position-order
+        // mode: per slot of the group, cached tokens (rl) and the live flag (ro); per row, its slot (rs) and visible prefix (rp).
+        int rl0[kRounds], ro0[kRounds], rs0[ORDER ? kRounds : 1], rp0[ORDER ? kRounds : 1];
+        auto load_tab = [&](int w, const WorkItem& it, int das, int dss, int dse, int* rl, int* ro, int* rs, int* rp) {
 #pragma unroll
             for (int r = 0; r < kRounds; ++r) {
                 const int b = lane + 32 * r;
                 rl[r] = 0; ro[r] = 0;
-                if (w < n_units && it.with_suffix && b < it.row_count) {
-                    const int row = das + it.row_begin + b;
-                    rl[r] = p.a.suffix_len[row];
-                    ro[r] = p.a.suffix_off[row];
+                if constexpr (ORDER) {
+                    rs[r] = -1; rp[r] = 0;
+                    if (w < n_units && b < it.row_count) {
+                        const int row = das + it.row_begin + b;
+                        rs[r] = p.a.active_slot[row];
+                        rp[r] = p.a.prefix_vis[row];
+                    }
+                    if (w < n_units && it.with_suffix && b < dse - dss) {
+                        rl[r] = p.a.slot_depth[dss + b];
+                        ro[r] = p.a.slot_alive[dss + b];
+                    }
+                } else {
+                    if (w < n_units && it.with_suffix && b < it.row_count) {
+                        const int row = das + it.row_begin + b;
+                        rl[r] = p.a.suffix_len[row];
+                        ro[r] = p.a.suffix_off[row];
+                    }
                 }
             }
         };
-        load_tab(w0, it0, das0, rl0, ro0);
+        load_tab(w0, it0, das0, dss0, dse0, rl0, ro0, rs0, rp0);
         uint32_t qc = 0, kc = 0, vc = 0;
         bool ok = true;
         for (uint32_t ui = 0; ok; ++ui) {
@@ -385,8 +417,10 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             const int w4 = static_cast<int>(ui) + 4 < kStatic ? fixed(static_cast<int>(ui) + 4) : draw();
             const WorkItem it3 = item_of(w3);
             const int das2 = p.a.doc_active_start[it2.doc], dks2 = p.a.doc_kv_start[it2.doc];
-            int rl1[kRounds], ro1[kRounds];
-            load_tab(w1, it1, das1, rl1, ro1);
+            int dss2 = 0, dse2 = 0;
+            if constexpr (ORDER) { dss2 = p.a.doc_slot_start[it2.doc]; dse2 = p.a.doc_slot_start[it2.doc + 1]; }
+            int rl1[kRounds], ro1[kRounds], rs1[ORDER ? kRounds : 1], rp1[ORDER ? kRounds : 1];
+            load_tab(w1, it1, das1, dss1, dse1, rl1, ro1, rs1, rp1);
             // ---- finish unit i: clamp, validate, scan, publish ----
             if (ui >= 1) {                               // the pipeline's consumers have copied the previous descriptor
                 ok = mbar_wait_warp(&misc->desc_empty[x], (ui - 1) & 1, misc);
@@ -395,17 +429,39 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             const bool live = w0 < n_units;
             int cs[kRounds], len[kRounds], off[kRounds];
             int carry = 0, bad = 0;
+            int nbr = 0;                                 // position-order mode: slots of the group the unit's rows may see
+            if constexpr (ORDER) {
+                int last = -1;                           // index in the group of the unit's last row's slot
+#pragma unroll
+                for (int r = 0; r < kRounds; ++r) {
+                    const int b = lane + 32 * r;
+                    const int idx = (live && b < it0.row_count) ? rs0[r] - dss0 : -1;
+                    if (b == it0.row_count - 1) last = idx;
+                    if (live && b < it0.row_count && (idx < 0 || idx >= kM || idx >= dse0 - dss0)) bad = 1;   // group too large or bad table
+                    d.ridx[b] = static_cast<uint16_t>(idx < 0 || idx >= kM ? 0 : idx);
+                    d.pvis[b] = (live && b < it0.row_count) ? rp0[r] - it0.key_begin : 0;
+                }
+                last = __reduce_max_sync(0xffffffffu, last);
+                nbr = (live && it0.with_suffix && last < kM) ? last + 1 : 0;
+            }
 #pragma unroll
             for (int r = 0; r < kRounds; ++r) {
                 const int b = lane + 32 * r;
                 int n = 0, o = 0;
-                if (live && it0.with_suffix && b < it0.row_count) {
+                if constexpr (ORDER) {
+                    if (b < nbr) {
+                        n = rl0[r] + (ro0[r] ? p.a.suffix_extra : 0);
+                        n = n < 0 ? 0 : (n > p.a.g.suffix_cap ? p.a.g.suffix_cap : n);
+                        const int64_t o64 = static_cast<int64_t>(dss0 + b) * p.a.g.suffix_cap;
+                        if (o64 + n > cache_rows) { bad = 1; n = 0; } else { o = static_cast<int>(o64); }
+                    }
+                } else if (live && it0.with_suffix && b < it0.row_count) {
                     n = rl0[r] + p.a.suffix_extra;
                     n = n < 0 ? 0 : (n > p.a.g.suffix_cap ? p.a.g.suffix_cap : n);
                     o = ro0[r];
                     if (o < 0 || static_cast<int64_t>(o) + n > cache_rows) { bad = 1; n = 0; o = 0; }
                 }
-                const int np4 = (n + kPad - 1) & ~(kPad - 1);        // columns the branch occupies
+                const int np4 = (n + PAD - 1) & ~(PAD - 1);          // columns the branch occupies
                 int incl = np4;
 #pragma unroll
                 for (int s = 1; s < 32; s <<= 1) {
@@ -438,7 +494,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     const int ks = kc % C::NK;
                     ok = mbar_wait_warp(&misc->k_empty[x][ks], ((kc / C::NK) & 1) ^ 1, misc);
                     if (!ok) break;
-                    fill_tile<D, false>(u, t, cs, len, off, lane, k_ring + ks * C::KV_BYTES, &misc->k_full[x][ks], &map_k, smaps.k);
+                    fill_tile<D, false, PAD>(u, t, cs, len, off, lane, k_ring + ks * C::KV_BYTES, &misc->k_full[x][ks], &map_k, smaps.k);
                     ++kc;
                     if (t == 0) {
                         // The Q tile is asked for after the unit's first K tile: its buffer is released late in the
@@ -457,7 +513,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     const int vs = vc % C::NV;
                     ok = mbar_wait_warp(&misc->v_empty[x][vs], ((vc / C::NV) & 1) ^ 1, misc);
                     if (!ok) break;
-                    fill_tile<D, true>(u, t - 1, cs, len, off, lane, v_ring + vs * C::KV_BYTES, &misc->v_full[x][vs], &map_v, smaps.v);
+                    fill_tile<D, true, PAD>(u, t - 1, cs, len, off, lane, v_ring + vs * C::KV_BYTES, &misc->v_full[x][vs], &map_v, smaps.v);
                     ++vc;
                 }
                 __syncwarp();
@@ -466,8 +522,12 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             w0 = w1; w1 = w2; w2 = w3; w3 = w4;
             it0 = it1; it1 = it2; it2 = it3;
             das0 = das1; dks0 = dks1; das1 = das2; dks1 = dks2;
+            if constexpr (ORDER) { dss0 = dss1; dse0 = dse1; dss1 = dss2; dse1 = dse2; }
 #pragma unroll
-            for (int r = 0; r < kRounds; ++r) { rl0[r] = rl1[r]; ro0[r] = ro1[r]; }
+            for (int r = 0; r < kRounds; ++r) {
+                rl0[r] = rl1[r]; ro0[r] = ro1[r];
+                if constexpr (ORDER) { rs0[r] = rs1[r]; rp0[r] = rp1[r]; }
+            }
         }
         }
     } else if (warp < 3) {
@@ -566,8 +626,17 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             ok = mbar_wait_warp(&misc->desc_full[x], unit_idx & 1, misc);
             if (!ok) break;
             const Unit u = read_unit(misc->desc[x]);
-            // packed columns [my_cs, my_cs + my_len) hold this row's own cached tokens
-            const int my_cs = misc->desc[x].cs[b_row], my_len = misc->desc[x].len[b_row];
+            // branch-local mode: packed columns [my_cs, my_cs + my_len) hold this row's own cached tokens.  Position-order
+            // mode: the row sees packed columns [0, my_cs + my_len) -- every slot up to its own -- and my_pv prefix tokens.
+            int my_cs, my_len, my_pv = 0;
+            if constexpr (ORDER) {
+                const int ri = min(static_cast<int>(misc->desc[x].ridx[min(b_row, kM - 1)]), kM - 1);
+                my_cs = 0;
+                my_len = misc->desc[x].cs[ri] + misc->desc[x].len[ri];
+                my_pv = misc->desc[x].pvis[min(b_row, kM - 1)];
+            } else {
+                my_cs = misc->desc[x].cs[b_row]; my_len = misc->desc[x].len[b_row];
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(&misc->desc_empty[x]);
             if (u.nt < 0) break;
@@ -583,7 +652,8 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 if (warp_active) {
                     const int ns = nt - u.np;
                     if (j >= ns) {
-                        hi = min(kN, u.key_count - (j - ns) * kN);
+                        hi = min(kN, (ORDER ? min(u.key_count, my_pv) : u.key_count) - (j - ns) * kN);
+                        if (hi < 0) hi = 0;
                     } else {
                         const int base = j * kN;
                         lo = max(0, my_cs - base);
@@ -856,15 +926,16 @@ bool make_q_map(CUtensorMap* m, const void* base, int D, int G, int Hkv, long lo
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D>
+template <int D, bool ORDER>
 int launch_d(const AttnArgs& a)
 {
     using C = Cfg<D>;
+    using SufMaps = SufMapsT<ORDER ? 16 : kBoxKinds>;
     // the dynamic shared-memory limit is an attribute of the kernel on ONE device: set it once per device
     static std::atomic<bool> attr_set[kMaxDevices];
     const int dev = current_device();
     if (dev < 0 || dev >= kMaxDevices || !attr_set[dev].load(std::memory_order_acquire)) {
-        HPD_CUDA_TRY(cudaFuncSetAttribute(hpd_attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
+        HPD_CUDA_TRY(cudaFuncSetAttribute(hpd_attn_tc_kernel<D, ORDER>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
         if (dev >= 0 && dev < kMaxDevices) attr_set[dev].store(true, std::memory_order_release);
     }
     const int G = a.g.Hq / a.g.Hkv;
@@ -895,7 +966,8 @@ int launch_d(const AttnArgs& a)
         ms->valid = false;
         bool maps_ok = make_q_map(&ms->mq, a.q, D, G, a.g.Hkv, a.max_rows) && make_kv_map(&ms->mk, kbase, D, a.g.Hkv, a.total_prefix, kN) &&
                        make_kv_map(&ms->mv, vbase, D, a.g.Hkv, a.total_prefix, kN);
-        for (int i = 0; i < kBoxKinds && maps_ok; ++i) maps_ok = make_kv_map(&ms->sm.k[i], a.suffix_k, D, a.g.Hkv, cache_rows, 4 * (i + 1));
+        for (int i = 0; i < (ORDER ? 16 : kBoxKinds) && maps_ok; ++i)
+            maps_ok = make_kv_map(&ms->sm.k[i], a.suffix_k, D, a.g.Hkv, cache_rows, ORDER ? i + 1 : 4 * (i + 1));
         for (int i = 0; i < 16 && maps_ok; ++i) maps_ok = make_kv_map(&ms->sm.v[i], a.suffix_v, D, a.g.Hkv, cache_rows, i + 1);
         if (!maps_ok) {
             set_last_cuda_error(cudaErrorInvalidValue);
@@ -916,7 +988,7 @@ int launch_d(const AttnArgs& a)
     p.scale_log2 = a.g.sm_scale * kLog2e;
     p.G = G;
     const int n_sm = sm_count();
-    hpd_attn_tc_kernel<D><<<n_sm, kThreads, C::SMEM, a.stream>>>(mq, mk, mv, sm, p);
+    hpd_attn_tc_kernel<D, ORDER><<<n_sm, kThreads, C::SMEM, a.stream>>>(mq, mk, mv, sm, p);
     hpd_merge_kernel<D><<<n_sm * 2, 256, 0, a.stream>>>(p, reinterpret_cast<const DocSplit*>(ws + a.lay.off_split));
     HPD_CUDA_TRY(cudaGetLastError());
     return HPD_OK;
@@ -927,7 +999,8 @@ int launch_d(const AttnArgs& a)
 int launch_attn_tc(const AttnArgs& a)
 {
     if (!(a.g.sm_scale > 0.f)) return HPD_E_GEOM;
-    return a.g.D == 128 ? launch_d<128>(a) : launch_d<64>(a);
+    if (a.active_slot) return a.g.D == 128 ? launch_d<128, true>(a) : launch_d<64, true>(a);
+    return a.g.D == 128 ? launch_d<128, false>(a) : launch_d<64, false>(a);
 }
 
 }  // namespace hpd

@@ -92,6 +92,9 @@ struct AttnArgs {
     const __nv_bfloat16 *q, *prefix_k, *prefix_v, *suffix_k, *suffix_v;
     const int32_t *doc_kv_start, *doc_prefix_len, *doc_active_start, *doc_id, *suffix_off, *suffix_len, *n_active;
     int suffix_extra;                // 1: suffix_len+1 cached tokens are visible
+    // position-order mode only (all null otherwise): slot tables of the groups and the rows' visible prefix lengths
+    const int32_t *doc_slot_start, *active_slot, *slot_depth, *prefix_vis;
+    const uint8_t* slot_alive;
     __nv_bfloat16* o;
     float* lse;
     void* workspace;
@@ -120,7 +123,8 @@ int launch_build_meta(const hpd_geom& g, int n_docs, int n_slots, const int32_t*
                       int32_t pos_gap, int32_t* doc_kv_start, int32_t* doc_slot_start, int32_t* doc_active_start,
                       int32_t* active_slot, int32_t* doc_id, int32_t* branch_start, int32_t* pos_id,
                       int32_t* suffix_off, int32_t* suffix_len, int32_t* n_active, void* workspace,
-                      const WsLayout& lay, int n_sm, int32_t* dev_status, cudaStream_t stream);
+                      const WsLayout& lay, int n_sm, int32_t* dev_status, cudaStream_t stream,
+                      const int32_t* slot_vis = nullptr, int32_t* prefix_vis = nullptr);
 int launch_rope(const hpd_geom& g, int max_rows, const int32_t* n_active, const int32_t* pos_id,
                 __nv_bfloat16* q, __nv_bfloat16* k_new, cudaStream_t stream);
 int launch_kv_append(const hpd_geom& g, int max_rows, int n_slots, const int32_t* n_active, const int32_t* suffix_off,

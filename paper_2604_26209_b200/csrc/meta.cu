@@ -80,9 +80,11 @@ compact_kernel(int n_docs, int n_slots, int32_t suffix_cap, int32_t pos_gap,
                const int32_t* __restrict__ doc_prefix_len, const int32_t* __restrict__ doc_branch_cnt,
                const int32_t* __restrict__ doc_slot_start,
                const int32_t* __restrict__ slot_depth, const uint8_t* __restrict__ slot_alive,
+               const int32_t* __restrict__ slot_vis /* nullable: anchor = document length */,
                int32_t* __restrict__ doc_active_start, int32_t* __restrict__ active_slot,
                int32_t* __restrict__ doc_id, int32_t* __restrict__ branch_start, int32_t* __restrict__ pos_id,
-               int32_t* __restrict__ suffix_off, int32_t* __restrict__ suffix_len, int32_t* __restrict__ n_active)
+               int32_t* __restrict__ suffix_off, int32_t* __restrict__ suffix_len,
+               int32_t* __restrict__ prefix_vis /* nullable */, int32_t* __restrict__ n_active)
 {
     __shared__ int sm[kCompactThreads / 32 + 1];
     const int first = blockIdx.x * kCompactThreads;
@@ -133,13 +135,15 @@ compact_kernel(int n_docs, int n_slots, int32_t suffix_cap, int32_t pos_gap,
         }
         if (alive) {
             const int depth = slot_depth[s];
-            const int bs = doc_prefix_len[d] + j * pos_gap;
+            const int anchor = slot_vis ? slot_vis[s] : doc_prefix_len[d];
+            const int bs = anchor + j * pos_gap;
             active_slot[excl] = s;
             doc_id[excl] = d;
             branch_start[excl] = bs;
             pos_id[excl] = bs + depth;
             suffix_off[excl] = s * suffix_cap;
             suffix_len[excl] = depth;
+            if (prefix_vis) prefix_vis[excl] = anchor;
         }
     }
     if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) {
@@ -281,6 +285,7 @@ plan_kernel(int n_docs, int n_slots, int G, int Hkv, int n_sm,
             const int32_t* __restrict__ n_active,
             int32_t* __restrict__ active_slot, int32_t* __restrict__ doc_id, int32_t* __restrict__ branch_start,
             int32_t* __restrict__ pos_id, int32_t* __restrict__ suffix_off, int32_t* __restrict__ suffix_len,
+            int32_t* __restrict__ prefix_vis /* nullable */,
             WsHeader* __restrict__ hdr, WorkItem* __restrict__ work, DocSplit* __restrict__ split,
             int work_cap, int part_cap)
 {
@@ -290,6 +295,7 @@ plan_kernel(int n_docs, int n_slots, int G, int Hkv, int n_sm,
         for (int i = na + (blockIdx.x - 1) * kPlanThreads + threadIdx.x; i < n_slots; i += (gridDim.x - 1) * kPlanThreads) {
             active_slot[i] = -1; doc_id[i] = -1; branch_start[i] = -1;
             pos_id[i] = -1; suffix_off[i] = -1; suffix_len[i] = -1;
+            if (prefix_vis) prefix_vis[i] = -1;
         }
         return;
     }
@@ -329,9 +335,11 @@ __global__ void __launch_bounds__(kFusedThreads)
 meta_fused_kernel(int n_docs, int n_slots, int32_t suffix_cap, int32_t pos_gap, int G, int Hkv, int n_sm,
                   const int32_t* __restrict__ doc_prefix_len, const int32_t* __restrict__ doc_branch_cnt,
                   const int32_t* __restrict__ slot_depth, const uint8_t* __restrict__ slot_alive,
+                  const int32_t* __restrict__ slot_vis /* nullable */,
                   int32_t* __restrict__ doc_kv_start, int32_t* __restrict__ doc_slot_start, int32_t* doc_active_start,
                   int32_t* __restrict__ active_slot, int32_t* __restrict__ doc_id, int32_t* __restrict__ branch_start,
                   int32_t* __restrict__ pos_id, int32_t* __restrict__ suffix_off, int32_t* __restrict__ suffix_len,
+                  int32_t* __restrict__ prefix_vis /* nullable */,
                   int32_t* __restrict__ n_active, WsHeader* hdr, WorkItem* __restrict__ work, DocSplit* __restrict__ split,
                   int work_cap, int part_cap)
 {
@@ -391,17 +399,20 @@ meta_fused_kernel(int n_docs, int n_slots, int32_t suffix_cap, int32_t pos_gap, 
         }
         if (alive) {
             const int depth = slot_depth[s];
-            const int bs = doc_prefix_len[d] + j * pos_gap;
+            const int anchor = slot_vis ? slot_vis[s] : doc_prefix_len[d];
+            const int bs = anchor + j * pos_gap;
             active_slot[excl] = s;
             doc_id[excl] = d;
             branch_start[excl] = bs;
             pos_id[excl] = bs + depth;
             suffix_off[excl] = s * suffix_cap;
             suffix_len[excl] = depth;
+            if (prefix_vis) prefix_vis[excl] = anchor;
         } else {
             const int t = total + (s - excl);            // the dead slots fill the tail of every row table with -1
             active_slot[t] = -1; doc_id[t] = -1; branch_start[t] = -1;
             pos_id[t] = -1; suffix_off[t] = -1; suffix_len[t] = -1;
+            if (prefix_vis) prefix_vis[t] = -1;
         }
     }
     if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) {
@@ -448,7 +459,8 @@ int launch_build_meta(const hpd_geom& g, int n_docs, int n_slots, const int32_t*
                       int32_t pos_gap, int32_t* doc_kv_start, int32_t* doc_slot_start, int32_t* doc_active_start,
                       int32_t* active_slot, int32_t* doc_id, int32_t* branch_start, int32_t* pos_id,
                       int32_t* suffix_off, int32_t* suffix_len, int32_t* n_active, void* workspace,
-                      const WsLayout& lay, int n_sm, int32_t* /*dev_status*/, cudaStream_t stream)
+                      const WsLayout& lay, int n_sm, int32_t* /*dev_status*/, cudaStream_t stream,
+                      const int32_t* slot_vis, int32_t* prefix_vis)
 {
     char* ws = static_cast<char*>(workspace);
     WsHeader* hdr = reinterpret_cast<WsHeader*>(ws);
@@ -462,8 +474,8 @@ int launch_build_meta(const hpd_geom& g, int n_docs, int n_slots, const int32_t*
         const int blocks = n_slots > 0 ? (n_slots + kFusedThreads - 1) / kFusedThreads : 1;
         meta_fused_kernel<<<blocks, kFusedThreads, 0, stream>>>(
             n_docs, n_slots, g.suffix_cap, pos_gap, g.Hq / g.Hkv, g.Hkv, n_sm, doc_prefix_len, doc_branch_cnt, slot_depth,
-            slot_alive, doc_kv_start, doc_slot_start, doc_active_start, active_slot, doc_id, branch_start, pos_id,
-            suffix_off, suffix_len, n_active, hdr, work, split, lay.work_cap, lay.part_cap);
+            slot_alive, slot_vis, doc_kv_start, doc_slot_start, doc_active_start, active_slot, doc_id, branch_start, pos_id,
+            suffix_off, suffix_len, prefix_vis, n_active, hdr, work, split, lay.work_cap, lay.part_cap);
         HPD_CUDA_TRY(cudaGetLastError());
         return HPD_OK;
     }
@@ -471,13 +483,13 @@ int launch_build_meta(const hpd_geom& g, int n_docs, int n_slots, const int32_t*
     const int cblocks = n_slots > 0 ? (n_slots + kCompactThreads - 1) / kCompactThreads : 1;
     compact_kernel<<<cblocks, kCompactThreads, 0, stream>>>(
         n_docs, n_slots, g.suffix_cap, pos_gap, doc_prefix_len, doc_branch_cnt, doc_slot_start, slot_depth, slot_alive,
-        doc_active_start, active_slot, doc_id, branch_start, pos_id, suffix_off, suffix_len, n_active);
+        slot_vis, doc_active_start, active_slot, doc_id, branch_start, pos_id, suffix_off, suffix_len, prefix_vis, n_active);
     int fill_blocks = (n_slots + kPlanThreads * 4 - 1) / (kPlanThreads * 4);
     if (fill_blocks < 1) fill_blocks = 1;
     if (fill_blocks > 64) fill_blocks = 64;
     plan_kernel<<<1 + fill_blocks, kPlanThreads, 0, stream>>>(
         n_docs, n_slots, g.Hq / g.Hkv, g.Hkv, n_sm, doc_prefix_len, doc_active_start, n_active, active_slot, doc_id,
-        branch_start, pos_id, suffix_off, suffix_len, hdr, work, split, lay.work_cap, lay.part_cap);
+        branch_start, pos_id, suffix_off, suffix_len, prefix_vis, hdr, work, split, lay.work_cap, lay.part_cap);
     HPD_CUDA_TRY(cudaGetLastError());
     return HPD_OK;
 }

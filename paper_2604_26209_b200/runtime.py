@@ -38,6 +38,7 @@ class DeviceBatch:
         self.prefix_v = _bf16(t["prefix_v"], device) if s.total_prefix else torch.zeros(8, dtype=torch.bfloat16, device=device)
         self.suffix_k = _bf16(t["suffix_k"], device) if s.n_slots else torch.zeros(8, dtype=torch.bfloat16, device=device)
         self.suffix_v = _bf16(t["suffix_v"], device) if s.n_slots else torch.zeros(8, dtype=torch.bfloat16, device=device)
+        self.slot_vis = i32(s.slot_vis) if (s.slot_vis is not None and s.n_slots) else None     # position-order workloads
         self.meta = B.MetaTables.alloc(self.g, s.n_docs, s.n_slots, s.total_prefix, device)
         n = max(s.n_slots, 1)
         self.q = torch.zeros(n, self.g.Hq, self.g.D, dtype=torch.bfloat16, device=device)
@@ -49,6 +50,10 @@ class DeviceBatch:
     # -- the C-ABI calls, in the order of one step -------------------------------------------
     def build_meta(self):
         s = self.s
+        if self.slot_vis is not None:
+            B.hpd_build_meta_skeleton(self.g, s.n_docs, s.n_slots, self.doc_prefix_len, self.doc_branch_cnt, self.slot_depth,
+                                      self.slot_alive, self.slot_vis, s.pos_gap, self.meta)
+            return
         B.hpd_build_meta(self.g, s.n_docs, s.n_slots, self.doc_prefix_len, self.doc_branch_cnt, self.slot_depth,
                          self.slot_alive, s.pos_gap, self.meta)
 
@@ -74,6 +79,11 @@ class DeviceBatch:
 
     def attn(self, suffix_includes_new=True, lse=True):
         s = self.s
+        if self.slot_vis is not None:
+            B.hpd_attn_decode_posorder(self.g, s.n_docs, s.n_slots, s.n_slots, s.total_prefix, self.q, self.prefix_k,
+                                       self.prefix_v, self.suffix_k, self.suffix_v, self.doc_prefix_len, self.slot_depth,
+                                       self.slot_alive, self.meta, suffix_includes_new, self.o, self.lse if lse else None)
+            return
         B.hpd_attn_decode(self.g, s.n_docs, s.n_slots, s.n_slots, s.total_prefix, self.q, self.prefix_k, self.prefix_v,
                           self.suffix_k, self.suffix_v, self.doc_prefix_len, self.meta, suffix_includes_new, self.o,
                           self.lse if lse else None)
@@ -102,7 +112,8 @@ class DeviceBatch:
     def tables(self) -> Dict[str, np.ndarray]:
         s = self.s
         out = {}
-        for name in B.MetaTables.NAMES:
+        names = B.MetaTables.NAMES + (("prefix_vis",) if self.slot_vis is not None else ())
+        for name in names:
             a = getattr(self.meta, name).cpu().numpy()
             n = s.n_docs + 1 if name.startswith("doc_") and name != "doc_id" else s.n_slots
             out[name] = a[:n].copy()
