@@ -158,6 +158,20 @@ int hpd_attn_decode(const hpd_geom* geom /*host*/, int n_docs, int max_rows, int
                     void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream);
 
 /*
+ * hpd_advance -- the end of a decode step on the device (Sec. 4.3.4 "Early Stopping"; the prune of
+ * Algorithm 1), so that the loop needs no host round trip per step.  token_id[r] is the token sampled
+ * from row r's output.  For every row r < *n_active with slot s = active_slot[r]:
+ *   slot_depth[s] = min(slot_depth[s] + 1, suffix_cap)      the step's input token is in the cache now
+ *   slot_alive[s] = 0 if token_id[r] == delimiter_id        (the value is complete: its delimiter came)
+ *                     or slot_depth[s] == suffix_cap        (K_max reached: the value is truncated)
+ * and n_alive[0] (dev) = number of rows that stay alive: generation ends when it reaches 0.  The next
+ * hpd_build_meta reads the updated slot tables.  token_id [max_rows] int32 dev.
+ */
+int hpd_advance(const hpd_geom* geom /*host*/, int max_rows, const int32_t* n_active, const int32_t* active_slot,
+                const int32_t* token_id, int32_t delimiter_id, int32_t* slot_depth, uint8_t* slot_alive,
+                int32_t* n_alive, void* stream);
+
+/*
  * Position-order mode: the mask the paper's implementation runs (Sec. 4.3.2: "the triangular attention
  * mask is computed using the position ID ordering"; Fig. 3; Sec. 4.4; Algorithm 2).  A "document" of the
  * tables is then a whole stacked prompt: its prefix is the prompt followed by the skeleton, i.e. the

@@ -24,6 +24,7 @@ def lib():
         _lib.hpdo_build_meta.restype = C.c_int
         _lib.hpdo_alg2_value_position.restype = C.c_int32
         _lib.hpdo_build_meta_skeleton.restype = C.c_int
+        _lib.hpdo_advance.restype = C.c_int
         _lib.hpdo_decode_step_posorder.restype = C.c_int
     return _lib
 
@@ -217,3 +218,13 @@ def decode_step_posorder(geom, meta: Meta, doc_prefix_len, slot_depth, slot_aliv
     if used < 0:
         raise MemoryError("oracle decode_step_posorder: allocation failed")
     return StepOut(o, lse, q_rot, k_rot, used), pos[:n]
+
+
+def advance(meta: Meta, token_id, delimiter: int, k_max: int, slot_depth: np.ndarray, slot_alive: np.ndarray) -> int:
+    """End of a step (Sec. 4.3.4), in place on int32 ``slot_depth`` / uint8 ``slot_alive``; returns rows still alive."""
+    assert slot_depth.dtype == np.int32 and slot_alive.dtype == np.uint8
+    n = meta.n_active
+    act, tok = _i32(meta.active_slot[:n]), _i32(token_id)
+    assert len(tok) >= n
+    return int(lib().hpdo_advance(C.c_int(n), _p(act), _p(tok), C.c_int32(delimiter), C.c_int32(k_max),
+                                  _p(slot_depth), _p(slot_alive)))

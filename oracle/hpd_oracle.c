@@ -440,3 +440,23 @@ int hpdo_decode_step_posorder(int Hq, int Hkv, int D, double theta, double scale
     free(pos); free(kr);
     return fail ? -1 : used;
 }
+
+/* ------------------------------------------------------------------------------------
+ * End of a decode step (Sec. 4.3.4, the prune of Algorithm 1).  tok[r] is the token sampled for
+ * live row r.  The step's input token has been appended, so the slot's depth grows by one (a full
+ * slab stays full); the value is finished when its delimiter was sampled, and truncated when the
+ * slab -- K_max tokens -- is full.  Returns the number of rows that stay alive; generation ends
+ * when it is 0 ("every value is pruned") or, through the second rule, after K_max steps.
+ * ---------------------------------------------------------------------------------- */
+int hpdo_advance(int n_active, const int32_t* active_slot, const int32_t* tok, int32_t delimiter,
+                 int32_t k_max, int32_t* slot_depth, uint8_t* slot_alive)
+{
+    int stay = 0;
+    for (int r = 0; r < n_active; ++r) {
+        int s = active_slot[r];
+        if (slot_depth[s] < k_max) slot_depth[s] += 1;
+        if (tok[r] == delimiter || slot_depth[s] >= k_max) slot_alive[s] = 0;
+        else { slot_alive[s] = 1; ++stay; }
+    }
+    return stay;
+}

@@ -173,6 +173,19 @@ int hpd_rope_append(const hpd_geom* geom, int max_rows, int n_slots, const int32
                               static_cast<__nv_bfloat16*>(suffix_v), dev_status, static_cast<cudaStream_t>(stream));
 }
 
+int hpd_advance(const hpd_geom* geom, int max_rows, const int32_t* n_active, const int32_t* active_slot,
+                const int32_t* token_id, int32_t delimiter_id, int32_t* slot_depth, uint8_t* slot_alive,
+                int32_t* n_alive, void* stream)
+{
+    int rc = geom_check(geom);
+    if (rc != HPD_OK) return rc;
+    if (max_rows < 0) return HPD_E_ARG;
+    if (!n_alive) return HPD_E_ARG;
+    if (max_rows > 0 && (!n_active || !active_slot || !token_id || !slot_depth || !slot_alive)) return HPD_E_ARG;
+    return launch_advance(*geom, max_rows, n_active, active_slot, token_id, delimiter_id, slot_depth, slot_alive, n_alive,
+                          static_cast<cudaStream_t>(stream));
+}
+
 struct OrderTables {                 // extra tables of the position-order mode (all null in the branch-local mode)
     const int32_t *doc_slot_start, *active_slot, *slot_depth, *prefix_vis;
     const uint8_t* slot_alive;

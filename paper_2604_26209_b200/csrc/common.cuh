@@ -134,6 +134,9 @@ int launch_rope_append(const hpd_geom& g, int max_rows, int n_slots, const int32
                        const int32_t* suffix_off, const int32_t* suffix_len, __nv_bfloat16* q, __nv_bfloat16* k_new,
                        const __nv_bfloat16* v_new, __nv_bfloat16* suffix_k, __nv_bfloat16* suffix_v, int32_t* dev_status,
                        cudaStream_t stream);
+int launch_advance(const hpd_geom& g, int max_rows, const int32_t* n_active, const int32_t* active_slot,
+                   const int32_t* token_id, int32_t delimiter_id, int32_t* slot_depth, uint8_t* slot_alive,
+                   int32_t* n_alive, cudaStream_t stream);
 int launch_attn_std(const StdArgs& a);         // TMA ring + warp-level tensor-core instructions
 int launch_attn_tc(const AttnArgs& a);       // tcgen05 / TMA kernel
 

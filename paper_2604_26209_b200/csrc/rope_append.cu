@@ -133,7 +133,39 @@ kv_append_kernel(int row_u4 /* Hkv*D*2/16 */, int32_t suffix_cap, int64_t cache_
     }
 }
 
+// End of a decode step (Sec. 4.3.4): one thread per row.
+__global__ void __launch_bounds__(256)
+advance_kernel(int max_rows, int32_t suffix_cap, int32_t delimiter_id, const int32_t* __restrict__ n_active,
+               const int32_t* __restrict__ active_slot, const int32_t* __restrict__ token_id,
+               int32_t* __restrict__ slot_depth, uint8_t* __restrict__ slot_alive, int32_t* __restrict__ n_alive)
+{
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    const int n = min(*n_active, max_rows);
+    int stays = 0;
+    if (r < n) {
+        const int s = active_slot[r];
+        const int d = min(slot_depth[s] + 1, suffix_cap);          // the step's token went into the slab (unless it was full)
+        slot_depth[s] = d;
+        stays = token_id[r] != delimiter_id && d < suffix_cap;
+        slot_alive[s] = static_cast<uint8_t>(stays);
+    }
+    const int cnt = __syncthreads_count(stays);
+    if (threadIdx.x == 0 && cnt) atomicAdd(n_alive, cnt);
+}
+
 }  // namespace
+
+int launch_advance(const hpd_geom& g, int max_rows, const int32_t* n_active, const int32_t* active_slot,
+                   const int32_t* token_id, int32_t delimiter_id, int32_t* slot_depth, uint8_t* slot_alive,
+                   int32_t* n_alive, cudaStream_t stream)
+{
+    HPD_CUDA_TRY(cudaMemsetAsync(n_alive, 0, sizeof(int32_t), stream));
+    if (max_rows <= 0) return HPD_OK;
+    advance_kernel<<<(max_rows + 255) / 256, 256, 0, stream>>>(max_rows, g.suffix_cap, delimiter_id, n_active, active_slot,
+                                                                token_id, slot_depth, slot_alive, n_alive);
+    HPD_CUDA_TRY(cudaGetLastError());
+    return HPD_OK;
+}
 
 int launch_rope(const hpd_geom& g, int max_rows, const int32_t* n_active, const int32_t* pos_id,
                 __nv_bfloat16* q, __nv_bfloat16* k_new, cudaStream_t stream)

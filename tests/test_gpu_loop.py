@@ -152,3 +152,49 @@ def test_fullsize_loop_two_layers_sampled_branches():
             ck = cache_k[l][lo:lo + m]
             assert np.all(np.abs(gk[lo:lo + m] - ck) <= np.abs(ck) * 2.0 ** -8 + 1e-6)
             assert np.array_equal(gv[lo:lo + m], cache_v[l][lo:lo + m])
+
+
+def test_device_side_retirement_drives_the_loop():
+    """Algorithm 1 for steps t >= 1 without a host round trip per step: hpd_advance turns the sampled token ids into
+    slot_alive / slot_depth on the device (Sec. 4.3.4), the next hpd_build_meta reads them.  The sampler is a stand-in:
+    a table of token ids per (step, slot) with the delimiter where the value ends, gathered by row with a torch index op.
+    Row counts of every step and the final slot tables must equal the oracle's loop, bit for bit."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2604_26209_b200 import binding as B
+    s0 = synth.config_loop(n_prompts=2, seed=9, mean_len=5, cap=12)
+    g, dev, delim = s0.geom, "cuda", 3
+    rng = np.random.default_rng(1)
+    K = np.minimum(rng.geometric(1.0 / 5, size=s0.n_slots), 20).astype(np.int32)      # some values longer than K_max = 12
+    steps = g.suffix_cap + 1
+    tok_tab = np.full((steps, s0.n_slots), 17, np.int32)
+    for sl in range(s0.n_slots):
+        if K[sl] - 1 < steps:
+            tok_tab[K[sl] - 1, sl] = delim                             # the token sampled at step K-1 ends the value
+    tb = synth.make_tensors(s0)
+    from paper_2604_26209_b200 import runtime
+    db = runtime.DeviceBatch(s0, tb)
+    db.slot_depth.zero_(); db.slot_alive.fill_(1)
+    tok_dev = torch.from_numpy(tok_tab).to(dev)
+    n_alive = torch.zeros(1, dtype=torch.int32, device=dev)
+    hist = torch.zeros(steps, 2, dtype=torch.int32, device=dev)
+    db.set_step_inputs(tb["q"], tb["k_new"], tb["v_new"])
+    for t in range(steps):
+        db.build_meta()
+        rows_tok = tok_dev[t][db.meta.active_slot.clamp(min=0).long()].contiguous()
+        db.rope_append()
+        db.attn(True, lse=False)
+        B.hpd_advance(g, s0.n_slots, db.meta.n_active, db.meta.active_slot, rows_tok, delim, db.slot_depth, db.slot_alive, n_alive)
+        hist[t, 0].copy_(db.meta.n_active[0]); hist[t, 1].copy_(n_alive[0])
+    torch.cuda.synchronize()
+    assert db.status() == 0
+    # the oracle's loop
+    depth, alive = np.zeros(s0.n_slots, np.int32), np.ones(s0.n_slots, np.uint8)
+    want = np.zeros((steps, 2), np.int32)
+    for t in range(steps):
+        meta = capi.build_meta(s0.doc_prefix_len, s0.doc_branch_cnt, depth, alive, g.suffix_cap, 0)
+        stay = capi.advance(meta, tok_tab[t][meta.active_slot[: meta.n_active]], delim, g.suffix_cap, depth, alive) if meta.n_active else 0
+        want[t] = (meta.n_active, stay)
+    assert np.array_equal(hist.cpu().numpy(), want)
+    assert np.array_equal(db.slot_depth.cpu().numpy(), depth) and np.array_equal(db.slot_alive.cpu().numpy(), alive)
+    assert np.array_equal(depth, np.minimum(K, g.suffix_cap)) and want[-1, 0] == 0     # everything pruned or truncated at K_max

@@ -122,3 +122,36 @@ def test_retired_and_empty():
     assert m.n_active == 0 and m.doc_kv_start.tolist() == [0]
     with pytest.raises(ValueError):
         capi.build_meta([4], [3], [0, 0], [1, 1], 4, 0)      # branch counts do not add up
+
+
+def test_advance_prunes_on_delimiter_and_truncates_at_k_max():
+    """Sec. 4.3.4 on a hand-written case: K_max = 3, delimiter 9.  Slots 0..4; slot 3 is already retired."""
+    depth = np.array([0, 2, 1, 1, 2], np.int32)
+    alive = np.array([1, 1, 1, 0, 1], np.uint8)
+    meta = capi.build_meta([5], [5], depth, alive, 3, 0)
+    assert list(meta.active_slot[:4]) == [0, 1, 2, 4]
+    stay = capi.advance(meta, [7, 7, 9, 9], 9, 3, depth, alive)
+    # slot 0: 0 -> 1, goes on; slot 1: 2 -> 3 = K_max, truncated although no delimiter came; slot 2: delimiter;
+    # slot 3: untouched; slot 4: delimiter (and full)
+    assert list(depth) == [1, 3, 2, 1, 3] and list(alive) == [1, 0, 0, 0, 0] and stay == 1
+
+
+def test_loop_ends_when_all_values_are_pruned_or_after_k_max_steps():
+    """Algorithm 1's loop with the prune rule: a value of K tokens is alive for exactly min(K, K_max) steps, its slab ends
+    up holding min(K, K_max) tokens, and the loop stops by itself after max(min(K, K_max)) <= K_max steps."""
+    rng = np.random.default_rng(4)
+    k_max, delim = 6, 0
+    K = rng.integers(1, 11, size=40)                                   # value lengths, some longer than K_max
+    depth, alive = np.zeros(40, np.int32), np.ones(40, np.uint8)
+    steps = 0
+    while True:
+        meta = capi.build_meta([3, 9], [15, 25], depth, alive, k_max, 0)
+        if meta.n_active == 0:
+            break
+        assert steps < k_max
+        act = meta.active_slot[: meta.n_active]
+        assert np.array_equal(act, np.nonzero(np.minimum(K, k_max) > steps)[0])
+        tok = np.where(depth[act] + 1 == K[act], delim, 5)             # the token sampled at this step
+        capi.advance(meta, tok, delim, k_max, depth, alive)
+        steps += 1
+    assert steps == int(np.minimum(K, k_max).max()) and np.array_equal(depth, np.minimum(K, k_max))
