@@ -25,6 +25,7 @@ def lib():
         _lib.hpdo_alg2_value_position.restype = C.c_int32
         _lib.hpdo_build_meta_skeleton.restype = C.c_int
         _lib.hpdo_advance.restype = C.c_int
+        _lib.hpdo_decode_step_shared3.restype = C.c_int
         _lib.hpdo_decode_step_posorder.restype = C.c_int
     return _lib
 
@@ -228,3 +229,41 @@ def advance(meta: Meta, token_id, delimiter: int, k_max: int, slot_depth: np.nda
     assert len(tok) >= n
     return int(lib().hpdo_advance(C.c_int(n), _p(act), _p(tok), C.c_int32(delimiter), C.c_int32(k_max),
                                   _p(slot_depth), _p(slot_alive)))
+
+
+def decode_step_shared3(geom, meta: Meta, doc_prefix_len, doc_block, block_len, q, k_new, v_new, block_k, block_v,
+                        prefix_k, prefix_v, suffix_k, suffix_v, n_threads: int = 0):
+    """One decode step with three sharing levels (Sec. 4.3.5): block ``doc_block[d]`` of ``block_len`` tokens precedes
+    document d.  ``meta`` are the ordinary tables of the documents.  Returns (StepOut, positions)."""
+    n = meta.n_active
+    q, k_new, v_new = _f32(q), _f32(k_new), _f32(v_new)
+    blk, bl = _i32(doc_block), _i32(block_len)
+    bstart = _i32(np.concatenate([[0], np.cumsum(bl)])[:-1])
+    L = _i32(doc_prefix_len)
+    did, soff, slen = _i32(meta.doc_id[:n]), _i32(meta.suffix_off[:n]), _i32(meta.suffix_len[:n])
+    block_k, block_v, prefix_k, prefix_v = _f32(block_k), _f32(block_v), _f32(prefix_k), _f32(prefix_v)
+    suffix_k, suffix_v = _f32(suffix_k), _f32(suffix_v)
+    o = np.empty((n, geom.Hq, geom.D), dtype=np.float32)
+    lse = np.empty((n, geom.Hq), dtype=np.float32)
+    q_rot = np.empty((n, geom.Hq, geom.D), dtype=np.float32)
+    k_rot = np.empty((n, geom.Hkv, geom.D), dtype=np.float32)
+    pos = np.empty(max(n, 1), dtype=np.int32)
+    used = lib().hpdo_decode_step_shared3(
+        C.c_int(geom.Hq), C.c_int(geom.Hkv), C.c_int(geom.D), C.c_double(geom.rope_theta), C.c_double(geom.sm_scale),
+        C.c_int(n), _p(did), _p(blk), _p(bstart), _p(bl), _p(soff), _p(slen), _p(meta.doc_kv_start), _p(L),
+        _p(q), _p(k_new), _p(v_new), _p(block_k), _p(block_v), _p(prefix_k), _p(prefix_v), _p(suffix_k), _p(suffix_v),
+        _p(o), _p(lse), _p(q_rot), _p(k_rot), _p(pos), C.c_int(n_threads))
+    if used < 0:
+        raise MemoryError("oracle decode_step_shared3: allocation failed")
+    return StepOut(o, lse, q_rot, k_rot, used), pos[:n]
+
+
+def merge_lse(o_a, lse_a, o_b, lse_b):
+    """Combine two attention results over disjoint key sets; arrays [..., D] and [...]."""
+    o_a = np.ascontiguousarray(o_a, dtype=np.float64); o_b = np.ascontiguousarray(o_b, dtype=np.float64)
+    la = np.ascontiguousarray(lse_a, dtype=np.float64); lb = np.ascontiguousarray(lse_b, dtype=np.float64)
+    D = o_a.shape[-1]
+    n = la.size
+    o = np.empty_like(o_a); lse = np.empty_like(la)
+    lib().hpdo_merge_lse(C.c_int(n), C.c_int(D), _p(o_a), _p(la), _p(o_b), _p(lb), _p(o), _p(lse))
+    return o, lse

@@ -460,3 +460,95 @@ int hpdo_advance(int n_active, const int32_t* active_slot, const int32_t* tok, i
     }
     return stay;
 }
+
+/* ====================================================================================
+ * Three sharing levels (Sec. 4.3.5: "the instruction and attribute definition is efficiently shared
+ * among all documents"): a block of tokens common to several documents, then the document, then the
+ * branch.  The sequence of a branch is [block ; document ; own tokens ; new token] at positions
+ * 0, 1, 2, ...; its output is ordinary causal attention at the last index, exactly as if the block
+ * had been stored in front of every document.
+ * ==================================================================================== */
+int hpdo_decode_step_shared3(int Hq, int Hkv, int D, double theta, double scale,
+                             int n_active, const int32_t* doc_id, const int32_t* doc_block,
+                             const int32_t* block_kv_start, const int32_t* block_len,
+                             const int32_t* suffix_off, const int32_t* suffix_len,
+                             const int32_t* doc_kv_start, const int32_t* doc_prefix_len,
+                             const float* q, const float* k_new, const float* v_new,
+                             const float* block_k, const float* block_v,
+                             const float* prefix_k, const float* prefix_v,
+                             const float* suffix_k, const float* suffix_v,
+                             float* o, float* lse, float* q_rot, float* k_rot, int32_t* pos_out, int n_threads)
+{
+    int used = 1, fail = 0;
+    size_t kvw = (size_t)Hkv * D, qw = (size_t)Hq * D;
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#endif
+#pragma omp parallel
+    {
+#ifdef _OPENMP
+#pragma omp single
+        used = omp_get_num_threads();
+#endif
+#pragma omp for schedule(dynamic, 1)
+        for (int r = 0; r < n_active; ++r) {
+            int d = doc_id[r], b = doc_block[d];
+            int LB = block_len[b], L = doc_prefix_len[d], k = suffix_len[r];
+            int n = LB + L + k + 1;
+            int pos = LB + L + k;
+            double* Kc = (double*)malloc(sizeof(double) * (size_t)n * kvw);
+            double* Vc = (double*)malloc(sizeof(double) * (size_t)n * kvw);
+            double* qr = (double*)malloc(sizeof(double) * qw);
+            double* orow = (double*)malloc(sizeof(double) * qw);
+            double* lrow = (double*)malloc(sizeof(double) * (size_t)Hq);
+            double* sc = (double*)malloc(sizeof(double) * (size_t)n);
+            if (!Kc || !Vc || !qr || !orow || !lrow || !sc) {
+                fail = 1;
+            } else {
+                size_t at = 0;
+                const float* bk = block_k + (size_t)block_kv_start[b] * kvw;
+                const float* bv = block_v + (size_t)block_kv_start[b] * kvw;
+                for (size_t i = 0; i < (size_t)LB * kvw; ++i) { Kc[at + i] = bk[i]; Vc[at + i] = bv[i]; }
+                at += (size_t)LB * kvw;
+                const float* pk = prefix_k + (size_t)doc_kv_start[d] * kvw;
+                const float* pv = prefix_v + (size_t)doc_kv_start[d] * kvw;
+                for (size_t i = 0; i < (size_t)L * kvw; ++i) { Kc[at + i] = pk[i]; Vc[at + i] = pv[i]; }
+                at += (size_t)L * kvw;
+                const float* sk = suffix_k + (size_t)suffix_off[r] * kvw;
+                const float* sv = suffix_v + (size_t)suffix_off[r] * kvw;
+                for (size_t i = 0; i < (size_t)k * kvw; ++i) { Kc[at + i] = sk[i]; Vc[at + i] = sv[i]; }
+                at += (size_t)k * kvw;
+                hpdo_rope(Hkv, D, theta, pos, k_new + (size_t)r * kvw, Kc + at);
+                for (size_t i = 0; i < kvw; ++i) Vc[at + i] = v_new[(size_t)r * kvw + i];
+                hpdo_rope(Hq, D, theta, pos, q + (size_t)r * qw, qr);
+                hpdo_causal_attention_row(n - 1, Hq, Hkv, D, scale, qr, Kc, Vc, orow, lrow, sc);
+                for (size_t i = 0; i < qw; ++i) o[(size_t)r * qw + i] = (float)orow[i];
+                if (lse) for (int h = 0; h < Hq; ++h) lse[(size_t)r * Hq + h] = (float)lrow[h];
+                if (q_rot) for (size_t i = 0; i < qw; ++i) q_rot[(size_t)r * qw + i] = (float)qr[i];
+                if (k_rot) for (size_t i = 0; i < kvw; ++i) k_rot[(size_t)r * kvw + i] = (float)Kc[at + i];
+                if (pos_out) pos_out[r] = pos;
+            }
+            free(Kc); free(Vc); free(qr); free(orow); free(lrow); free(sc);
+        }
+    }
+    return fail ? -1 : used;
+}
+
+/* Two attention results over disjoint key sets, each a normalised output with the log-sum-exp of
+ * its scores, combined into the result over the union: weights e^{lse_a} and e^{lse_b}. */
+void hpdo_merge_lse(int n, int D, const double* o_a, const double* lse_a, const double* o_b, const double* lse_b,
+                    double* o, double* lse)
+{
+    for (int i = 0; i < n; ++i) {
+        double m = lse_a[i] > lse_b[i] ? lse_a[i] : lse_b[i];
+        if (m == -INFINITY) {
+            for (int d = 0; d < D; ++d) o[(size_t)i * D + d] = 0.0;
+            lse[i] = -INFINITY;
+            continue;
+        }
+        double wa = exp(lse_a[i] - m), wb = exp(lse_b[i] - m);
+        for (int d = 0; d < D; ++d)
+            o[(size_t)i * D + d] = (wa * o_a[(size_t)i * D + d] + wb * o_b[(size_t)i * D + d]) / (wa + wb);
+        lse[i] = m + log(wa + wb);
+    }
+}
