@@ -172,6 +172,22 @@ int hpd_advance(const hpd_geom* geom /*host*/, int max_rows, const int32_t* n_ac
                 int32_t* n_alive, void* stream);
 
 /*
+ * hpd_merge_lse -- three sharing levels (Sec. 4.3.5: the instruction and the attribute definitions are
+ * shared among all documents).  A block of tokens common to several documents is attended ONCE per block
+ * for all rows below it by a second hpd_attn_decode call whose "documents" are the blocks (tables from a
+ * second hpd_build_meta over the blocks, its own workspace, an all-zero suffix_len table and
+ * suffix_includes_new = 0, the block's K/V as prefix); this call combines the two results per (row, head):
+ *     o = (e^{lse_a} o_a + e^{lse_b} o_b) / (e^{lse_a} + e^{lse_b}),   lse = log(e^{lse_a} + e^{lse_b}).
+ * Both calls need their lse outputs.  o may alias o_a or o_b, lse may alias lse_a or lse_b or be NULL.
+ * Position IDs then count the block too: build the document tables with hpd_build_meta_skeleton,
+ * slot_vis = block length + L_d and pos_gap = 0.
+ *   o_a, o_b, o [max_rows, Hq, D] bf16 dev; lse_a, lse_b, lse [max_rows, Hq] fp32 dev.
+ */
+int hpd_merge_lse(const hpd_geom* geom /*host*/, int max_rows, const int32_t* n_active,
+                  const void* o_a, const float* lse_a, const void* o_b, const float* lse_b,
+                  void* o, float* lse, void* stream);
+
+/*
  * Position-order mode: the mask the paper's implementation runs (Sec. 4.3.2: "the triangular attention
  * mask is computed using the position ID ordering"; Fig. 3; Sec. 4.4; Algorithm 2).  A "document" of the
  * tables is then a whole stacked prompt: its prefix is the prompt followed by the skeleton, i.e. the
@@ -185,7 +201,8 @@ int hpd_advance(const hpd_geom* geom /*host*/, int max_rows, const int32_t* n_ac
  * hpd_build_meta_skeleton -- hpd_build_meta with a per-slot anchor:
  *   slot_vis[n_slots] (dev)   prefix tokens of the slot's group up to and including its attribute key
  *                             (= end(a_j) + 1 in Algorithm 2's notation; 0 <= slot_vis <= L_d, ascending
- *                             inside a group)
+ *                             inside a group).  The builder only uses it as the position anchor of the
+ *                             slot's first token; hpd_merge_lse's three-level layout passes a larger one.
  *   branch_start[r] = slot_vis + j*pos_gap   (= pos_id[end(a_j)] + 1 of Algorithm 2)
  *   prefix_vis[r]   = slot_vis of the row's slot (n_slots entries, -1 past n_active)
  * Everything else as hpd_build_meta.

@@ -18,7 +18,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libhpd.so")
 
 EXPORTS = ("hpd_strerror", "hpd_last_cuda_error", "hpd_workspace_bytes", "hpd_build_meta", "hpd_rope",
-           "hpd_kv_append", "hpd_rope_append", "hpd_attn_decode", "hpd_build_meta_skeleton", "hpd_attn_decode_posorder", "hpd_advance", "std_workspace_bytes", "std_attn_decode",
+           "hpd_kv_append", "hpd_rope_append", "hpd_attn_decode", "hpd_build_meta_skeleton", "hpd_attn_decode_posorder", "hpd_advance", "hpd_merge_lse", "std_workspace_bytes", "std_attn_decode",
            "std_attn_decode_static_max_bytes", "std_attn_decode_static")
 
 HPD_S_OVERFLOW, HPD_S_BAD_TABLE, HPD_S_TIMEOUT = 1, 2, 4
@@ -60,6 +60,8 @@ def load() -> C.CDLL:
         lib.hpd_attn_decode_posorder.restype = C.c_int
         lib.hpd_attn_decode_posorder.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int, C.c_int, C.c_int] + [vp] * 15 + \
                                                 [C.c_int, vp, vp, vp, C.c_size_t, vp, vp]
+        lib.hpd_merge_lse.restype = C.c_int
+        lib.hpd_merge_lse.argtypes = [C.POINTER(HpdGeom), C.c_int] + [vp] * 8
         lib.hpd_advance.restype = C.c_int
         lib.hpd_advance.argtypes = [C.POINTER(HpdGeom), C.c_int, vp, vp, vp, C.c_int32, vp, vp, vp, vp]
         lib.hpd_rope.restype = C.c_int
@@ -176,6 +178,13 @@ def hpd_attn_decode_posorder(geom, n_docs, max_rows, n_slots, total_prefix_token
                                          _ptr(m.prefix_vis), _ptr(m.n_active), int(bool(suffix_includes_new)), _ptr(o),
                                          _ptr(lse), _ptr(m.workspace), m.workspace.numel(), _ptr(m.dev_status), _stream())
     _check(rc, "hpd_attn_decode_posorder")
+
+
+def hpd_merge_lse(geom, max_rows, n_active, o_a, lse_a, o_b, lse_b, o, lse=None):
+    g = make_geom(geom)
+    rc = load().hpd_merge_lse(C.byref(g), max_rows, _ptr(n_active), _ptr(o_a), _ptr(lse_a), _ptr(o_b), _ptr(lse_b), _ptr(o),
+                              _ptr(lse), _stream())
+    _check(rc, "hpd_merge_lse")
 
 
 def hpd_advance(geom, max_rows, n_active, active_slot, token_id, delimiter_id, slot_depth, slot_alive, n_alive):

@@ -186,6 +186,20 @@ int hpd_advance(const hpd_geom* geom, int max_rows, const int32_t* n_active, con
                           static_cast<cudaStream_t>(stream));
 }
 
+int hpd_merge_lse(const hpd_geom* geom, int max_rows, const int32_t* n_active, const void* o_a, const float* lse_a,
+                  const void* o_b, const float* lse_b, void* o, float* lse, void* stream)
+{
+    int rc = geom_check(geom);
+    if (rc != HPD_OK) return rc;
+    if (max_rows < 0) return HPD_E_ARG;
+    if (max_rows == 0) return HPD_OK;
+    if (!n_active || !o_a || !lse_a || !o_b || !lse_b || !o) return HPD_E_ARG;
+    if (!aligned16(o_a) || !aligned16(o_b) || !aligned16(o)) return HPD_E_ARG;
+    return launch_merge_lse(*geom, max_rows, n_active, static_cast<const __nv_bfloat16*>(o_a), lse_a,
+                            static_cast<const __nv_bfloat16*>(o_b), lse_b, static_cast<__nv_bfloat16*>(o), lse,
+                            static_cast<cudaStream_t>(stream));
+}
+
 struct OrderTables {                 // extra tables of the position-order mode (all null in the branch-local mode)
     const int32_t *doc_slot_start, *active_slot, *slot_depth, *prefix_vis;
     const uint8_t* slot_alive;

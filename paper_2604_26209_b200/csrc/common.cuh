@@ -137,6 +137,8 @@ int launch_rope_append(const hpd_geom& g, int max_rows, int n_slots, const int32
 int launch_advance(const hpd_geom& g, int max_rows, const int32_t* n_active, const int32_t* active_slot,
                    const int32_t* token_id, int32_t delimiter_id, int32_t* slot_depth, uint8_t* slot_alive,
                    int32_t* n_alive, cudaStream_t stream);
+int launch_merge_lse(const hpd_geom& g, int max_rows, const int32_t* n_active, const __nv_bfloat16* o_a, const float* lse_a,
+                     const __nv_bfloat16* o_b, const float* lse_b, __nv_bfloat16* o, float* lse, cudaStream_t stream);
 int launch_attn_std(const StdArgs& a);         // TMA ring + warp-level tensor-core instructions
 int launch_attn_tc(const AttnArgs& a);       // tcgen05 / TMA kernel
 

@@ -153,7 +153,54 @@ advance_kernel(int max_rows, int32_t suffix_cap, int32_t delimiter_id, const int
     if (threadIdx.x == 0 && cnt) atomicAdd(n_alive, cnt);
 }
 
+// Merge of two attention results over disjoint key sets (three-level sharing): one warp per (row, q head).
+template <int D>
+__global__ void __launch_bounds__(256)
+merge_lse_kernel(int Hq, int max_rows, const int32_t* __restrict__ n_active,
+                 const __nv_bfloat16* o_a, const float* lse_a, const __nv_bfloat16* o_b, const float* lse_b,
+                 __nv_bfloat16* o, float* lse)
+{
+    constexpr int E = D / 32;
+    const int lane = threadIdx.x & 31;
+    const int64_t w = static_cast<int64_t>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+    if (w >= static_cast<int64_t>(min(*n_active, max_rows)) * Hq) return;
+    const float la = lse_a[w], lb = lse_b[w];
+    const float m = fmaxf(la, lb);
+    float wa = 0.f, wb = 0.f, out_l = -INFINITY;
+    if (m != -INFINITY) {
+        const float ea = __expf(la - m), eb = __expf(lb - m);
+        wa = ea / (ea + eb); wb = eb / (ea + eb);
+        out_l = m + __logf(ea + eb);
+    }
+    const __nv_bfloat16* pa = o_a + w * D + lane * E;
+    const __nv_bfloat16* pb = o_b + w * D + lane * E;
+    __nv_bfloat16* po = o + w * D + lane * E;
+    if constexpr (E == 4) {
+        const uint2 a = *reinterpret_cast<const uint2*>(pa), b = *reinterpret_cast<const uint2*>(pb);
+        uint2 r;
+        r.x = pack_bf16(wa * bf16lo(a.x) + wb * bf16lo(b.x), wa * bf16hi(a.x) + wb * bf16hi(b.x));
+        r.y = pack_bf16(wa * bf16lo(a.y) + wb * bf16lo(b.y), wa * bf16hi(a.y) + wb * bf16hi(b.y));
+        *reinterpret_cast<uint2*>(po) = r;
+    } else {
+        const uint32_t a = *reinterpret_cast<const uint32_t*>(pa), b = *reinterpret_cast<const uint32_t*>(pb);
+        *reinterpret_cast<uint32_t*>(po) = pack_bf16(wa * bf16lo(a) + wb * bf16lo(b), wa * bf16hi(a) + wb * bf16hi(b));
+    }
+    if (lse && lane == 0) lse[w] = out_l;
+}
+
 }  // namespace
+
+int launch_merge_lse(const hpd_geom& g, int max_rows, const int32_t* n_active, const __nv_bfloat16* o_a, const float* lse_a,
+                     const __nv_bfloat16* o_b, const float* lse_b, __nv_bfloat16* o, float* lse, cudaStream_t stream)
+{
+    if (max_rows <= 0) return HPD_OK;
+    const int64_t warps = static_cast<int64_t>(max_rows) * g.Hq;
+    const unsigned blocks = static_cast<unsigned>((warps + 7) / 8);
+    if (g.D == 128) merge_lse_kernel<128><<<blocks, 256, 0, stream>>>(g.Hq, max_rows, n_active, o_a, lse_a, o_b, lse_b, o, lse);
+    else merge_lse_kernel<64><<<blocks, 256, 0, stream>>>(g.Hq, max_rows, n_active, o_a, lse_a, o_b, lse_b, o, lse);
+    HPD_CUDA_TRY(cudaGetLastError());
+    return HPD_OK;
+}
 
 int launch_advance(const hpd_geom& g, int max_rows, const int32_t* n_active, const int32_t* active_slot,
                    const int32_t* token_id, int32_t delimiter_id, int32_t* slot_depth, uint8_t* slot_alive,

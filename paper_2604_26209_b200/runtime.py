@@ -26,8 +26,10 @@ def bits_of(t: torch.Tensor) -> np.ndarray:
 class DeviceBatch:
     """One layer's decode state of a synthetic batch on the GPU."""
 
-    def __init__(self, s: Structure, t: Dict[str, np.ndarray], device="cuda"):
+    def __init__(self, s: Structure, t: Dict[str, np.ndarray], device="cuda", posorder: Optional[bool] = None):
         self.s, self.g, self.device = s, s.geom, device
+        # a structure with per-slot anchors runs the position-order mask unless told that they are anchors only
+        self.posorder = (s.slot_vis is not None) if posorder is None else posorder
         i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
         self.doc_prefix_len = i32(s.doc_prefix_len) if s.n_docs else torch.zeros(1, dtype=torch.int32, device=device)
         self.doc_branch_cnt = i32(s.doc_branch_cnt) if s.n_docs else torch.zeros(1, dtype=torch.int32, device=device)
@@ -79,7 +81,7 @@ class DeviceBatch:
 
     def attn(self, suffix_includes_new=True, lse=True):
         s = self.s
-        if self.slot_vis is not None:
+        if self.posorder:
             B.hpd_attn_decode_posorder(self.g, s.n_docs, s.n_slots, s.n_slots, s.total_prefix, self.q, self.prefix_k,
                                        self.prefix_v, self.suffix_k, self.suffix_v, self.doc_prefix_len, self.slot_depth,
                                        self.slot_alive, self.meta, suffix_includes_new, self.o, self.lse if lse else None)
@@ -122,6 +124,53 @@ class DeviceBatch:
 
     def status(self) -> int:
         return int(self.meta.dev_status.item())
+
+
+class SharedBlockBatch:
+    """Three sharing levels (Sec. 4.3.5): blocks of tokens common to several documents, the documents, the branches.
+    Two hpd_attn_decode calls -- rows against their document and branch cache, rows against their block -- and
+    hpd_merge_lse.  ``doc_block[d]`` = block of document d (blocks cover consecutive documents), ``block_len[b]`` tokens,
+    ``block_k/v`` bf16 bits [sum block_len, Hkv, D]."""
+
+    def __init__(self, s: Structure, t: Dict[str, np.ndarray], doc_block: np.ndarray, block_len: np.ndarray,
+                 block_k: np.ndarray, block_v: np.ndarray, device="cuda"):
+        from dataclasses import replace
+        doc_block = np.asarray(doc_block, dtype=np.int64)
+        assert np.all(np.diff(doc_block) >= 0), "blocks cover consecutive documents"
+        self.n_blocks = int(len(block_len))
+        anchor = (np.asarray(block_len, np.int64)[doc_block] + s.doc_prefix_len)[s.slot_doc()].astype(np.int32)
+        self.db = DeviceBatch(replace(s, slot_vis=anchor, pos_gap=0), t, device, posorder=False)
+        g = s.geom
+        i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
+        cnt = np.zeros(self.n_blocks, np.int64)
+        np.add.at(cnt, doc_block, s.doc_branch_cnt)
+        self.block_len, self.block_cnt = i32(block_len), i32(cnt)
+        self.total_block = int(np.sum(block_len))
+        self.block_k = _bf16(block_k, device) if self.total_block else torch.zeros(8, dtype=torch.bfloat16, device=device)
+        self.block_v = _bf16(block_v, device) if self.total_block else torch.zeros(8, dtype=torch.bfloat16, device=device)
+        self.meta_b = B.MetaTables.alloc(g, self.n_blocks, s.n_slots, self.total_block, device)
+        zeros = torch.zeros(max(s.n_slots, 1), dtype=torch.int32, device=device)
+        self.meta_b_nosuffix = replace(self.meta_b, suffix_off=zeros, suffix_len=zeros)
+        self.o_b = torch.zeros_like(self.db.o)
+        self.lse_b = torch.zeros_like(self.db.lse)
+
+    def build_meta(self):
+        db, s = self.db, self.db.s
+        db.build_meta()
+        B.hpd_build_meta(self.db.g, self.n_blocks, s.n_slots, self.block_len, self.block_cnt, db.slot_depth, db.slot_alive, 0,
+                         self.meta_b)
+
+    def attn(self):
+        db, s, g = self.db, self.db.s, self.db.g
+        db.attn(True, lse=True)
+        B.hpd_attn_decode(g, self.n_blocks, s.n_slots, s.n_slots, self.total_block, db.q, self.block_k, self.block_v,
+                          db.suffix_k, db.suffix_v, self.block_len, self.meta_b_nosuffix, False, self.o_b, self.lse_b)
+        B.hpd_merge_lse(g, s.n_slots, db.meta.n_active, db.o, db.lse, self.o_b, self.lse_b, db.o, db.lse)
+
+    def step(self):
+        self.build_meta()
+        self.db.rope_append()
+        self.attn()
 
 
 class DupBatch:
