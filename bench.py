@@ -42,6 +42,8 @@ def workload_prompts(workload: str) -> int:
         return 32
     if workload.startswith("main_p"):
         return int(workload[6:])
+    if workload.startswith("long_p"):
+        return int(workload[6:])
     if workload.startswith("posorder_p"):
         return int(workload[10:])
     raise SystemExit(f"unknown workload {workload}")
@@ -55,7 +57,7 @@ def rank_structure(workload: str, world: int, rank: int):
     a one-rank run is the single-GPU workload itself.  Returns (structure, range of global prompt indices)."""
     per_gpu = workload_prompts(workload)
     mine = synth.shard_prompts(per_gpu * world, world, rank)
-    if workload == "long":
+    if workload.startswith("long"):
         s = synth.config_long(n_prompts=len(mine), seed=mine.start)
     elif workload.startswith("posorder_p"):
         # the mask the paper runs (Sec. 4.3.2): every prompt is ONE group -- 4 stacked documents of 512 tokens as the
