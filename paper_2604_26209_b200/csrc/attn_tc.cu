@@ -5,9 +5,9 @@
 // query heads, the M dimension) against a chunk of that document's prefix, so each prefix K/V byte
 // is read from HBM once for all of the document's branches.  Keys are consumed in tiles of 64:
 // first the tiles into which the branches' own cached tokens ("suffix") are packed back to back,
-// each branch padded to a multiple of four columns so that one TMA box of 4..16 cache rows places
-// it (the few K rows read beyond a branch's length are masked; V boxes have the exact height),
-// masked block-diagonally (a row sees only its own branch's columns); then the prefix tiles.  The
+// one TMA box of the exact height (1..16 cache rows) per branch and half of D, masked
+// block-diagonally (a row sees only its own branch's columns; in the position-order mode the
+// columns of every slot up to its own); then the prefix tiles.  The
 // suffix tiles come first because their many small copies are slow to issue and can be issued
 // while the pipeline's previous unit is still being finished.
 //
@@ -56,8 +56,6 @@ constexpr int kRegsIo = 104, kRegsSoftmax = 200;
 // setmaxnreg only moves registers inside the CTA's own allocation (168 x 384 threads at launch): a request beyond
 // that pool would block forever; using the pool exactly is fine
 static_assert(kRegsIo + 2 * kRegsSoftmax <= 3 * 168, "registers traded between the warpgroups exceed the CTA's allocation");
-constexpr int kBoxKinds = 4;               // suffix boxes of 4, 8, 12, 16 cache rows
-constexpr int kPad = 4;                    // a branch's cached tokens occupy a multiple of 4 packed columns
 constexpr int kRounds = 4;                 // a unit has at most 128 branches: 4 rounds of 32 lanes
 constexpr int kDescReaders = 5;            // readers of a pipeline's unit descriptor: its MMA thread and its four softmax warps
 constexpr int kMaxStages = 4;              // K or V stages of one pipeline (barrier storage)
@@ -78,9 +76,9 @@ template <int D> struct Cfg {
 };
 static_assert(Cfg<128>::SMEM <= 232448, "shared memory budget");
 
-template <int NK> struct SufMapsT {        // tensor maps of the branch cache, one per box height
-    CUtensorMap k[NK];                      // NK = 4: 4, 8, 12, 16 rows (padded packing); NK = 16: 1 .. 16 rows (exact)
-    CUtensorMap v[16];                      // 1 .. 16 rows
+struct SufMaps {                            // tensor maps of the branch cache, one per box height: 1 .. 16 rows
+    CUtensorMap k[16];
+    CUtensorMap v[16];
 };
 
 struct TcParams {
@@ -240,11 +238,10 @@ __device__ __forceinline__ Unit read_unit(const UnitDesc& d) {
 }
 
 // One K or V tile of a unit.  A prefix tile is two boxes issued by lane 0; a suffix tile is packed from one box per
-// branch (and half), every lane placing the part of its branches that falls into the tile.  K boxes are 4, 8, 12 or
-// 16 rows high and may read up to three rows past the branch's length (their columns are masked); V boxes (EXACT) have
-// the exact height, because whatever lies beyond a branch's length in the cache -- possibly NaN -- would otherwise be
-// multiplied by a zero probability.
-template <int D, bool EXACT, int PAD>
+// branch (and half), every lane placing the part of its branches that falls into the tile.  Boxes have the exact height
+// of the piece (tensor maps for 1..16 rows), so nothing beyond a branch's length is ever read: whatever lies there in
+// the cache -- possibly NaN -- must not meet a zero probability, and the packing needs no padding.
+template <int D>
 __device__ __forceinline__ void fill_tile(const Unit& u, int t, const int (&cs)[kRounds], const int (&len)[kRounds], const int (&off)[kRounds],
                                           int lane, uint8_t* tile, unsigned long long* full, const CUtensorMap* pre, const CUtensorMap* suf)
 {
@@ -261,21 +258,19 @@ __device__ __forceinline__ void fill_tile(const Unit& u, int t, const int (&cs)[
         int rows_mine = 0;
 #pragma unroll
         for (int r = 0; r < kRounds; ++r) {
-            const int plen = EXACT ? len[r] : (len[r] + PAD - 1) & ~(PAD - 1);
-            rows_mine += max(0, min(cs[r] + plen, c_hi) - max(cs[r], c_lo));
+            rows_mine += max(0, min(cs[r] + len[r], c_hi) - max(cs[r], c_lo));
         }
         const int rows_all = __reduce_add_sync(0xffffffffu, rows_mine);
         if (lane == 0) mbar_expect_tx(full, static_cast<uint32_t>(rows_all) * D * 2);
 #pragma unroll
         for (int r = 0; r < kRounds; ++r) {
-            const int plen = EXACT ? len[r] : (len[r] + PAD - 1) & ~(PAD - 1);
-            const int lo = max(cs[r], c_lo), hi = min(cs[r] + plen, c_hi);
+            const int lo = max(cs[r], c_lo), hi = min(cs[r] + len[r], c_hi);
             int n = hi - lo;
             int row = off[r] + (lo - cs[r]);
             int col = lo - c_lo;
             while (n > 0) {
                 const int hb = min(n, 16);
-                const CUtensorMap* m = (EXACT || PAD == 1) ? &suf[hb - 1] : &suf[hb / 4 - 1];
+                const CUtensorMap* m = &suf[hb - 1];
                 for (int h = 0; h < C::HALVES; ++h)
                     tma_load_3d(tile + h * kKHalf + col * 128, m, full, h * 64, u.head, row);
                 row += hb; col += hb; n -= hb;
@@ -291,15 +286,13 @@ __device__ __forceinline__ void fill_tile(const Unit& u, int t, const int (&cs)[
 // ORDER = true:  position-order mask (Sec. 4.3.2, Fig. 3): a group is a whole stacked prompt; a row sees the first
 //                prefix_vis[row] prefix tokens (prompt and the skeleton up to its own attribute key) and the cached
 //                tokens of every slot of the group up to and including its own -- live or retired --, which is "position
-//                ID not larger than mine" under Algorithm 2's K_max gaps.  Branch tokens are then packed without padding
-//                (K boxes of the exact height), so a row's visible packed columns are one range starting at 0.
+//                ID not larger than mine" under Algorithm 2's K_max gaps.  Branch tokens are packed back to back in slot
+//                order, so a row's visible packed columns are one range starting at 0.
 template <int D, bool ORDER>
 __global__ void __launch_bounds__(kThreads, 1)
 hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                   const __grid_constant__ CUtensorMap map_v, const __grid_constant__ SufMapsT<ORDER ? 16 : kBoxKinds> smaps,
-                   const TcParams p)
+                   const __grid_constant__ CUtensorMap map_v, const __grid_constant__ SufMaps smaps, const TcParams p)
 {
-    constexpr int PAD = ORDER ? 1 : kPad;
     using C = Cfg<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
     Misc* misc = reinterpret_cast<Misc*>(smem + C::OFF_MISC);
@@ -461,14 +454,13 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     o = ro0[r];
                     if (o < 0 || static_cast<int64_t>(o) + n > cache_rows) { bad = 1; n = 0; o = 0; }
                 }
-                const int np4 = (n + PAD - 1) & ~(PAD - 1);          // columns the branch occupies
-                int incl = np4;
+                int incl = n;                                // columns the branch occupies
 #pragma unroll
                 for (int s = 1; s < 32; s <<= 1) {
                     const int v = __shfl_up_sync(0xffffffffu, incl, s);
                     if (lane >= s) incl += v;
                 }
-                cs[r] = carry + incl - np4; len[r] = n; off[r] = o;
+                cs[r] = carry + incl - n; len[r] = n; off[r] = o;
                 d.cs[b] = static_cast<uint16_t>(cs[r]);
                 d.len[b] = static_cast<uint16_t>(n);
                 carry += __shfl_sync(0xffffffffu, incl, 31);
@@ -494,7 +486,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     const int ks = kc % C::NK;
                     ok = mbar_wait_warp(&misc->k_empty[x][ks], ((kc / C::NK) & 1) ^ 1, misc);
                     if (!ok) break;
-                    fill_tile<D, false, PAD>(u, t, cs, len, off, lane, k_ring + ks * C::KV_BYTES, &misc->k_full[x][ks], &map_k, smaps.k);
+                    fill_tile<D>(u, t, cs, len, off, lane, k_ring + ks * C::KV_BYTES, &misc->k_full[x][ks], &map_k, smaps.k);
                     ++kc;
                     if (t == 0) {
                         // The Q tile is asked for after the unit's first K tile: its buffer is released late in the
@@ -513,7 +505,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     const int vs = vc % C::NV;
                     ok = mbar_wait_warp(&misc->v_empty[x][vs], ((vc / C::NV) & 1) ^ 1, misc);
                     if (!ok) break;
-                    fill_tile<D, true, PAD>(u, t - 1, cs, len, off, lane, v_ring + vs * C::KV_BYTES, &misc->v_full[x][vs], &map_v, smaps.v);
+                    fill_tile<D>(u, t - 1, cs, len, off, lane, v_ring + vs * C::KV_BYTES, &misc->v_full[x][vs], &map_v, smaps.v);
                     ++vc;
                 }
                 __syncwarp();
@@ -930,7 +922,6 @@ template <int D, bool ORDER>
 int launch_d(const AttnArgs& a)
 {
     using C = Cfg<D>;
-    using SufMaps = SufMapsT<ORDER ? 16 : kBoxKinds>;
     // the dynamic shared-memory limit is an attribute of the kernel on ONE device: set it once per device
     static std::atomic<bool> attr_set[kMaxDevices];
     const int dev = current_device();
@@ -966,8 +957,7 @@ int launch_d(const AttnArgs& a)
         ms->valid = false;
         bool maps_ok = make_q_map(&ms->mq, a.q, D, G, a.g.Hkv, a.max_rows) && make_kv_map(&ms->mk, kbase, D, a.g.Hkv, a.total_prefix, kN) &&
                        make_kv_map(&ms->mv, vbase, D, a.g.Hkv, a.total_prefix, kN);
-        for (int i = 0; i < (ORDER ? 16 : kBoxKinds) && maps_ok; ++i)
-            maps_ok = make_kv_map(&ms->sm.k[i], a.suffix_k, D, a.g.Hkv, cache_rows, ORDER ? i + 1 : 4 * (i + 1));
+        for (int i = 0; i < 16 && maps_ok; ++i) maps_ok = make_kv_map(&ms->sm.k[i], a.suffix_k, D, a.g.Hkv, cache_rows, i + 1);
         for (int i = 0; i < 16 && maps_ok; ++i) maps_ok = make_kv_map(&ms->sm.v[i], a.suffix_v, D, a.g.Hkv, cache_rows, i + 1);
         if (!maps_ok) {
             set_last_cuda_error(cudaErrorInvalidValue);

@@ -31,8 +31,8 @@ int geom_check(const hpd_geom* g);   // HPD_OK or HPD_E_GEOM / HPD_E_ARG
 int current_device();                // ordinal of the calling thread's current device (0 if it cannot be queried)
 int sm_count();                      // SMs of the current device (148 if it cannot be queried)
 
-// hpd_attn_decode packs the cached tokens of the up to 128/G branches of a unit back to back, each branch rounded
-// up to a multiple of four columns, and stores a branch's first column and length as 16-bit numbers.
+// hpd_attn_decode packs the cached tokens of the up to 128/G branches of a unit back to back and stores a branch's
+// first column and length as 16-bit numbers (the limit is stated for slab sizes rounded up to a multiple of four).
 constexpr long long kMaxPackedColumns = 65535;
 inline long long attn_packed_columns(const hpd_geom& g)
 {
