@@ -544,7 +544,7 @@ def spawn_ranks(args) -> int:
 
 def run_loop(args):
     """Decode loop: 32 layers x up to 32 steps over the main structure with ragged retirement (end-of-value lengths
-    min(Geom(1/8), 32)).  Per step: hpd_build_meta once, then per layer hpd_rope -> hpd_kv_append -> hpd_attn_decode
+    min(Geom(1/8), 32)).  Per step: hpd_build_meta once, then per layer hpd_rope_append -> hpd_attn_decode
     on that layer's own prefix and branch caches.  Caches are filled on the device (torch.randn, seeded): 43 GB."""
     import torch
     from paper_2604_26209_b200 import binding as B
@@ -581,9 +581,8 @@ def run_loop(args):
         B.hpd_build_meta(g, s.n_docs, s.n_slots, L_d, cnt, depth, alive, 0, meta)
         for l in range(L):
             b = l & 1
-            B.hpd_rope(g, s.n_slots, meta.n_active, meta.pos_id, q[b], kn[b])
-            B.hpd_kv_append(g, s.n_slots, s.n_slots, meta.n_active, meta.suffix_off, meta.suffix_len, kn[b], vn[b],
-                            suf_k[l], suf_v[l], meta.dev_status)
+            B.hpd_rope_append(g, s.n_slots, s.n_slots, meta.n_active, meta.pos_id, meta.suffix_off, meta.suffix_len, q[b], kn[b],
+                              vn[b], suf_k[l], suf_v[l], meta.dev_status)
             B.hpd_attn_decode(g, s.n_docs, s.n_slots, s.n_slots, s.total_prefix, q[b], pre_k[l], pre_v[l], suf_k[l],
                               suf_v[l], L_d, meta, True, o, None)
 
@@ -620,7 +619,7 @@ def run_loop(args):
                                         "branches_per_prompt": 96, "suffix_cap": g.suffix_cap,
                                         "l2": "inputs larger than L2 (every layer has its own caches); no flush",
                                         "launch": "cuda graph replay of one decode step" if graph is not None else "direct calls"},
-        "clocks": clocks, "gpu_launches": steps * (3 + 4 * L), "dev_status": int(meta.dev_status.item()),
+        "clocks": clocks, "gpu_launches": steps * (1 + 3 * L), "dev_status": int(meta.dev_status.item()),
         "per_layer_branch_tokens_per_s": tokens * L / (total_ms * 1e-3),
         "series": [{"step": t, "n_active": n_act[t], "ms": ms[t]} for t in range(steps)],
     }))

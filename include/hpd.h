@@ -104,7 +104,8 @@ int hpd_build_meta(const hpd_geom* geom /*host*/, int n_docs, int n_slots,
  * hpd_rope -- rotary embedding of the step's new q and k at each row's position ID, in place
  * (Sec. 4.3.1: the assigned position IDs define the positional embedding; Sec. 4.4).
  * Pairing is half-split: element i with i + D/2; angle = pos_id[r] * rope_theta^(-2i/D),
- * evaluated in fp64, rotation in fp32, result rounded to bf16 (nearest even).
+ * taken and reduced to [-pi, pi] in fp64; sine, cosine and the rotation in fp32; result rounded to bf16
+ * (nearest even).
  *   q [max_rows, Hq, D] bf16 dev, k_new [max_rows, Hkv, D] bf16 dev; rows >= *n_active untouched.
  */
 int hpd_rope(const hpd_geom* geom /*host*/, int max_rows, const int32_t* n_active /*dev*/,

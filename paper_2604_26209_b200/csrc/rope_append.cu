@@ -13,10 +13,13 @@ namespace {
 
 constexpr int kRopeThreads = 256;
 
-// One CTA per row.  The row's D/2 (cos, sin) pairs are evaluated once in fp64 (angles reach
-// thousands of radians, where an fp32 product pos * inv_freq already loses ~1e-4 rad), kept in
-// shared memory as fp32, and applied to all Hq + Hkv heads: each thread rotates 8 pairs at a time
-// from one 16-byte load of the low half and one of the high half.
+// One CTA per row.  The row's D/2 (cos, sin) pairs are evaluated once, kept in shared memory as fp32 and applied to all
+// Hq + Hkv heads: each thread rotates 8 pairs at a time from one 16-byte load of the low half and one of the high half.
+// Angles reach thousands of radians, where an fp32 product pos * inv_freq already loses ~1e-4 rad: the product and its
+// reduction to [-pi, pi] are taken in fp64 (inverse frequencies computed in fp64 on the host, 2*pi split in two doubles),
+// and only the reduced angle goes through the fp32 sine and cosine.
+struct InvFreq { double f[64]; };                    // theta^(-2i/D), i < D/2 <= 64
+
 struct AppendDst {                                   // fused kernel only: where the row's key and value go
     int32_t suffix_cap;
     int64_t cache_rows;
@@ -28,7 +31,7 @@ struct AppendDst {                                   // fused kernel only: where
 
 template <int D, bool FUSED>
 __global__ void __launch_bounds__(kRopeThreads)
-rope_kernel(int Hq, int Hkv, double neg_log2_theta_2_over_d, const int32_t* __restrict__ n_active,
+rope_kernel(int Hq, int Hkv, const InvFreq inv_freq, const int32_t* __restrict__ n_active,
             const int32_t* __restrict__ pos_id, __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ k_new,
             const AppendDst ad)
 {
@@ -52,11 +55,14 @@ rope_kernel(int Hq, int Hkv, double neg_log2_theta_2_over_d, const int32_t* __re
         }
     }
     if (threadIdx.x < HALF) {
-        const double inv_freq = exp2(neg_log2_theta_2_over_d * static_cast<double>(threadIdx.x));
-        double s, c;
-        sincos(static_cast<double>(pos) * inv_freq, &s, &c);
-        cs[threadIdx.x] = static_cast<float>(c);
-        sn[threadIdx.x] = static_cast<float>(s);
+        const double ang = static_cast<double>(pos) * inv_freq.f[threadIdx.x];
+        const double k = rint(ang * 0.15915494309189535);                       // turns
+        double r = fma(-k, 6.283185307179586, ang);                             // minus k * 2*pi (high part, then the rest)
+        r = fma(-k, 2.4492935982947064e-16, r);
+        float s, c;
+        sincosf(static_cast<float>(r), &s, &c);
+        cs[threadIdx.x] = c;
+        sn[threadIdx.x] = s;
     }
     __syncthreads();
     const int items = (Hq + Hkv) * CHUNKS;
@@ -131,6 +137,13 @@ kv_append_kernel(int row_u4 /* Hkv*D*2/16 */, int32_t suffix_cap, int64_t cache_
         kd[i] = ks[i];
         vd[i] = vs[i];
     }
+}
+
+InvFreq inv_freq_table(const hpd_geom& g)
+{
+    InvFreq t{};
+    for (int i = 0; i < g.D / 2; ++i) t.f[i] = pow(static_cast<double>(g.rope_theta), -2.0 * i / static_cast<double>(g.D));
+    return t;
 }
 
 // End of a decode step (Sec. 4.3.4): one thread per row.
@@ -218,7 +231,7 @@ int launch_rope(const hpd_geom& g, int max_rows, const int32_t* n_active, const 
                 __nv_bfloat16* q, __nv_bfloat16* k_new, cudaStream_t stream)
 {
     if (max_rows <= 0) return HPD_OK;
-    const double c = -2.0 * log2(static_cast<double>(g.rope_theta)) / static_cast<double>(g.D);
+    const InvFreq c = inv_freq_table(g);
     const AppendDst none{};
     if (g.D == 128)
         rope_kernel<128, false><<<max_rows, kRopeThreads, 0, stream>>>(g.Hq, g.Hkv, c, n_active, pos_id, q, k_new, none);
@@ -234,7 +247,7 @@ int launch_rope_append(const hpd_geom& g, int max_rows, int n_slots, const int32
                        cudaStream_t stream)
 {
     if (max_rows <= 0) return HPD_OK;
-    const double c = -2.0 * log2(static_cast<double>(g.rope_theta)) / static_cast<double>(g.D);
+    const InvFreq c = inv_freq_table(g);
     const AppendDst ad{g.suffix_cap, static_cast<int64_t>(n_slots) * g.suffix_cap, suffix_off, suffix_len, v_new,
                        suffix_k, suffix_v, dev_status};
     if (g.D == 128)
