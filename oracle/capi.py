@@ -26,6 +26,7 @@ def lib():
         _lib.hpdo_build_meta_skeleton.restype = C.c_int
         _lib.hpdo_advance.restype = C.c_int
         _lib.hpdo_decode_step_shared3.restype = C.c_int
+        _lib.hpdo_prefill.restype = C.c_int
         _lib.hpdo_decode_step_posorder.restype = C.c_int
     return _lib
 
@@ -267,3 +268,23 @@ def merge_lse(o_a, lse_a, o_b, lse_b):
     o = np.empty_like(o_a); lse = np.empty_like(la)
     lib().hpdo_merge_lse(C.c_int(n), C.c_int(D), _p(o_a), _p(la), _p(o_b), _p(lb), _p(o), _p(lse))
     return o, lse
+
+
+def prefill(geom, doc_prefix_len, doc_branch_cnt, slot_vis, k_max: int, q, k, v, n_threads: int = 0):
+    """First inference step (Sec. 4.3.2): causal attention of every prompt token with Algorithm 2's position IDs.
+    ``q [T,Hq,D]``, ``k, v [T,Hkv,D]`` fp32 for the T prompt tokens.  Returns (StepOut over all T rows, positions [T])."""
+    L, cnt, vis = _i32(doc_prefix_len), _i32(doc_branch_cnt), _i32(slot_vis)
+    q, k, v = _f32(q), _f32(k), _f32(v)
+    T = int(L.sum())
+    assert q.shape == (T, geom.Hq, geom.D) and k.shape == (T, geom.Hkv, geom.D) and v.shape == k.shape
+    o = np.empty((T, geom.Hq, geom.D), dtype=np.float32)
+    lse = np.empty((T, geom.Hq), dtype=np.float32)
+    q_rot = np.empty((T, geom.Hq, geom.D), dtype=np.float32)
+    k_rot = np.empty((T, geom.Hkv, geom.D), dtype=np.float32)
+    pos = np.empty(max(T, 1), dtype=np.int32)
+    used = lib().hpdo_prefill(C.c_int(geom.Hq), C.c_int(geom.Hkv), C.c_int(geom.D), C.c_double(geom.rope_theta),
+                              C.c_double(geom.sm_scale), C.c_int(len(L)), _p(L), _p(cnt), _p(vis), C.c_int32(k_max),
+                              _p(q), _p(k), _p(v), _p(o), _p(lse), _p(q_rot), _p(k_rot), _p(pos), C.c_int(n_threads))
+    if used < 0:
+        raise MemoryError("oracle prefill: allocation failed")
+    return StepOut(o, lse, q_rot, k_rot, used), pos[:T]

@@ -552,3 +552,83 @@ void hpdo_merge_lse(int n, int D, const double* o_a, const double* lse_a, const 
         lse[i] = m + log(wa + wb);
     }
 }
+
+/* ====================================================================================
+ * First inference step (Sec. 4.3.2 "First Inference Step"; the prefill of Algorithm 1): the model
+ * input s = cat(p, a_1..a_N) of every group goes through ordinary causal attention -- in the
+ * prefill the memory order IS the position order -- with the rotary embedding taken at
+ * Algorithm 2's position IDs (a gap of K_max behind every attribute key).  The rotated keys and the
+ * values are what the decode steps later find in the prefix cache; the rows at the attribute ends
+ * are the ones whose outputs predict the first value tokens.
+ *   q [T,Hq,D], k,v [T,Hkv,D] for the T = sum L_d prompt tokens, groups back to back;
+ *   -> o [T,Hq,D], lse [T,Hq], k_rot [T,Hkv,D], q_rot [T,Hq,D], pos [T]   (fp32 outputs; may be NULL except o, pos)
+ * ==================================================================================== */
+int hpdo_prefill(int Hq, int Hkv, int D, double theta, double scale,
+                 int n_docs, const int32_t* doc_prefix_len, const int32_t* doc_branch_cnt, const int32_t* slot_vis,
+                 int32_t k_max,
+                 const float* q, const float* k, const float* v,
+                 float* o, float* lse, float* q_rot, float* k_rot, int32_t* pos, int n_threads)
+{
+    int used = 1, fail = 0;
+    size_t kvw = (size_t)Hkv * D, qw = (size_t)Hq * D;
+    /* position IDs: Algorithm 2 per group, attribute j spanning (end of j-1, end of j] */
+    {
+        int t0 = 0, s0 = 0;
+        for (int d = 0; d < n_docs; ++d) {
+            int L = doc_prefix_len[d], c = doc_branch_cnt[d];
+            int32_t* st = (int32_t*)malloc(sizeof(int32_t) * (size_t)(c > 0 ? c : 1));
+            int32_t* en = (int32_t*)malloc(sizeof(int32_t) * (size_t)(c > 0 ? c : 1));
+            if (!st || !en) { free(st); free(en); return -1; }
+            for (int j = 0; j < c; ++j) {
+                en[j] = slot_vis[s0 + j] - 1;
+                st[j] = j ? en[j - 1] + 1 : 0;
+            }
+            hpdo_alg2_position_ids(L, c, st, en, k_max, pos + t0);
+            free(st); free(en);
+            t0 += L; s0 += c;
+        }
+    }
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#endif
+    int t0 = 0;
+    for (int d = 0; d < n_docs; ++d) {
+        int L = doc_prefix_len[d];
+        double* Kc = (double*)malloc(sizeof(double) * (size_t)(L > 0 ? L : 1) * kvw);
+        double* Vc = (double*)malloc(sizeof(double) * (size_t)(L > 0 ? L : 1) * kvw);
+        if (!Kc || !Vc) { free(Kc); free(Vc); return -1; }
+        for (int t = 0; t < L; ++t) {
+            hpdo_rope(Hkv, D, theta, pos[t0 + t], k + (size_t)(t0 + t) * kvw, Kc + (size_t)t * kvw);
+            for (size_t i = 0; i < kvw; ++i) Vc[(size_t)t * kvw + i] = v[(size_t)(t0 + t) * kvw + i];
+            if (k_rot) for (size_t i = 0; i < kvw; ++i) k_rot[(size_t)(t0 + t) * kvw + i] = (float)Kc[(size_t)t * kvw + i];
+        }
+#pragma omp parallel
+        {
+#ifdef _OPENMP
+#pragma omp single
+            used = omp_get_num_threads();
+#endif
+            double* qr = (double*)malloc(sizeof(double) * qw);
+            double* orow = (double*)malloc(sizeof(double) * qw);
+            double* lrow = (double*)malloc(sizeof(double) * (size_t)Hq);
+            double* sc = (double*)malloc(sizeof(double) * (size_t)(L > 0 ? L : 1));
+            if (!qr || !orow || !lrow || !sc) {
+#pragma omp atomic write
+                fail = 1;
+            } else {
+#pragma omp for schedule(dynamic, 4)
+                for (int t = 0; t < L; ++t) {
+                    hpdo_rope(Hq, D, theta, pos[t0 + t], q + (size_t)(t0 + t) * qw, qr);
+                    hpdo_causal_attention_row(t, Hq, Hkv, D, scale, qr, Kc, Vc, orow, lrow, sc);
+                    for (size_t i = 0; i < qw; ++i) o[(size_t)(t0 + t) * qw + i] = (float)orow[i];
+                    if (lse) for (int h = 0; h < Hq; ++h) lse[(size_t)(t0 + t) * Hq + h] = (float)lrow[h];
+                    if (q_rot) for (size_t i = 0; i < qw; ++i) q_rot[(size_t)(t0 + t) * qw + i] = (float)qr[i];
+                }
+            }
+            free(qr); free(orow); free(lrow); free(sc);
+        }
+        free(Kc); free(Vc);
+        t0 += L;
+    }
+    return fail ? -1 : used;
+}
