@@ -232,6 +232,36 @@ int hpd_attn_decode_posorder(const hpd_geom* geom /*host*/, int n_docs, int max_
                              void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream);
 
 /*
+ * First inference step (Sec. 4.3.2 "First Inference Step"; the prefill of Algorithm 1): the whole model input
+ * s = cat(prompt, skeleton) of every group through causal attention -- in the prefill the memory order is the
+ * position order -- with the rotary embedding at Algorithm 2's position IDs.  Three calls:
+ *   hpd_prefill_meta   per prompt token x (T = sum L_d of them, groups back to back): tok_doc[x] its group,
+ *                      tok_pos[x] = t + pos_gap * #{slots of the group whose attribute key ends before t}
+ *                      (Algorithm 2 with start(a_j) = end(a_{j-1}) + 1), tok_vis[x] = t + 1 (its causal bound),
+ *                      t the token's index in its group; doc_kv_start, doc_slot_start; n_tokens[0] = T; and the
+ *                      attention's work list in `workspace` (hpd_workspace_bytes(geom, n_docs, total_tokens, ..)).
+ *                      At most 2048 groups per call (HPD_E_CAPACITY beyond).
+ *   hpd_rope           with max_rows = total_tokens, n_active = n_tokens, pos_id = tok_pos, q = the prompt
+ *                      tokens' queries and k_new = prefix_k itself: the keys are rotated in place in the prefix
+ *                      cache, where the decode steps find them; the values are stored unrotated by the caller.
+ *   hpd_prefill_attn   o[x] = causal attention of token x over its group's tokens 0..t; every 128/G tokens of a
+ *                      group form one tensor-core tile and visit only the keys up to the tile's last token.
+ * The rows that predict the first value tokens are those at the attribute ends, x = doc_kv_start[d] + slot_vis - 1
+ * ("decoded from positions 12, 22 and 32" in the paper's figure); when only they are needed (last layer),
+ * hpd_attn_decode_posorder on depth-0 slots with their queries does the same with 96 rows per prompt.
+ *   q, o [total_tokens, Hq, D] bf16; prefix_k, prefix_v [total_tokens, Hkv, D] bf16; lse [total_tokens, Hq] or NULL.
+ */
+int hpd_prefill_meta(const hpd_geom* geom /*host*/, int n_docs, int n_slots, int total_tokens,
+                     const int32_t* doc_prefix_len, const int32_t* doc_branch_cnt, const int32_t* slot_vis, int32_t pos_gap,
+                     int32_t* doc_kv_start, int32_t* doc_slot_start, int32_t* tok_doc, int32_t* tok_pos, int32_t* tok_vis,
+                     int32_t* n_tokens, void* workspace, size_t workspace_bytes, void* stream);
+int hpd_prefill_attn(const hpd_geom* geom /*host*/, int n_docs, int total_tokens,
+                     const void* q, const void* prefix_k, const void* prefix_v,
+                     const int32_t* doc_kv_start, const int32_t* doc_prefix_len, const int32_t* tok_doc, const int32_t* tok_vis,
+                     const int32_t* n_tokens, void* o, float* lse,
+                     void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream);
+
+/*
  * std_attn_decode -- the in-repo comparison: standard batched decode in which every branch is a
  * sequence of its own with a private physical copy of [prefix ; branch tokens] (parallel streams
  * as batch elements, Sec. 2; standard batched inference, Sec. 4.3.6).  Same math as

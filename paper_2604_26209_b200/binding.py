@@ -18,7 +18,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libhpd.so")
 
 EXPORTS = ("hpd_strerror", "hpd_last_cuda_error", "hpd_workspace_bytes", "hpd_build_meta", "hpd_rope",
-           "hpd_kv_append", "hpd_rope_append", "hpd_attn_decode", "hpd_build_meta_skeleton", "hpd_attn_decode_posorder", "hpd_advance", "hpd_merge_lse", "std_workspace_bytes", "std_attn_decode",
+           "hpd_kv_append", "hpd_rope_append", "hpd_attn_decode", "hpd_build_meta_skeleton", "hpd_attn_decode_posorder", "hpd_advance", "hpd_merge_lse", "hpd_prefill_meta", "hpd_prefill_attn", "std_workspace_bytes", "std_attn_decode",
            "std_attn_decode_static_max_bytes", "std_attn_decode_static")
 
 HPD_S_OVERFLOW, HPD_S_BAD_TABLE, HPD_S_TIMEOUT = 1, 2, 4
@@ -60,6 +60,11 @@ def load() -> C.CDLL:
         lib.hpd_attn_decode_posorder.restype = C.c_int
         lib.hpd_attn_decode_posorder.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int, C.c_int, C.c_int] + [vp] * 15 + \
                                                 [C.c_int, vp, vp, vp, C.c_size_t, vp, vp]
+        lib.hpd_prefill_meta.restype = C.c_int
+        lib.hpd_prefill_meta.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int, C.c_int, vp, vp, vp, C.c_int32] + [vp] * 6 + \
+                                        [vp, C.c_size_t, vp]
+        lib.hpd_prefill_attn.restype = C.c_int
+        lib.hpd_prefill_attn.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int] + [vp] * 10 + [vp, C.c_size_t, vp, vp]
         lib.hpd_merge_lse.restype = C.c_int
         lib.hpd_merge_lse.argtypes = [C.POINTER(HpdGeom), C.c_int] + [vp] * 8
         lib.hpd_advance.restype = C.c_int
@@ -178,6 +183,43 @@ def hpd_attn_decode_posorder(geom, n_docs, max_rows, n_slots, total_prefix_token
                                          _ptr(m.prefix_vis), _ptr(m.n_active), int(bool(suffix_includes_new)), _ptr(o),
                                          _ptr(lse), _ptr(m.workspace), m.workspace.numel(), _ptr(m.dev_status), _stream())
     _check(rc, "hpd_attn_decode_posorder")
+
+
+@dataclass
+class PrefillTables:
+    """Device tables of the first inference step (``hpd_prefill_meta``)."""
+    doc_kv_start: torch.Tensor
+    doc_slot_start: torch.Tensor
+    tok_doc: torch.Tensor
+    tok_pos: torch.Tensor
+    tok_vis: torch.Tensor
+    n_tokens: torch.Tensor
+    workspace: torch.Tensor
+    dev_status: torch.Tensor
+
+    @staticmethod
+    def alloc(geom, n_docs: int, total_tokens: int, device="cuda") -> "PrefillTables":
+        i32 = lambda n: torch.empty(max(n, 1), dtype=torch.int32, device=device)
+        ws = torch.empty(max(hpd_workspace_bytes(geom, n_docs, total_tokens, total_tokens), 256), dtype=torch.uint8, device=device)
+        return PrefillTables(i32(n_docs + 1), i32(n_docs + 1), i32(total_tokens), i32(total_tokens), i32(total_tokens),
+                             torch.zeros(1, dtype=torch.int32, device=device), ws, torch.zeros(1, dtype=torch.int32, device=device))
+
+
+def hpd_prefill_meta(geom, n_docs, n_slots, total_tokens, doc_prefix_len, doc_branch_cnt, slot_vis, pos_gap, t: PrefillTables):
+    g = make_geom(geom)
+    rc = load().hpd_prefill_meta(C.byref(g), n_docs, n_slots, total_tokens, _ptr(doc_prefix_len), _ptr(doc_branch_cnt),
+                                 _ptr(slot_vis), int(pos_gap), _ptr(t.doc_kv_start), _ptr(t.doc_slot_start), _ptr(t.tok_doc),
+                                 _ptr(t.tok_pos), _ptr(t.tok_vis), _ptr(t.n_tokens), _ptr(t.workspace), t.workspace.numel(),
+                                 _stream())
+    _check(rc, "hpd_prefill_meta")
+
+
+def hpd_prefill_attn(geom, n_docs, total_tokens, q, prefix_k, prefix_v, doc_prefix_len, t: PrefillTables, o, lse=None):
+    g = make_geom(geom)
+    rc = load().hpd_prefill_attn(C.byref(g), n_docs, total_tokens, _ptr(q), _ptr(prefix_k), _ptr(prefix_v),
+                                 _ptr(t.doc_kv_start), _ptr(doc_prefix_len), _ptr(t.tok_doc), _ptr(t.tok_vis), _ptr(t.n_tokens),
+                                 _ptr(o), _ptr(lse), _ptr(t.workspace), t.workspace.numel(), _ptr(t.dev_status), _stream())
+    _check(rc, "hpd_prefill_attn")
 
 
 def hpd_merge_lse(geom, max_rows, n_active, o_a, lse_a, o_b, lse_b, o, lse=None):

@@ -220,11 +220,12 @@ static int attn_common(const hpd_geom* geom, int n_docs, int max_rows, int n_slo
     if (attn_packed_columns(*geom) > kMaxPackedColumns) return HPD_E_CAPACITY;
     if (n_docs < 0 || max_rows < 0 || n_slots < 0 || total_prefix_tokens < 0) return HPD_E_ARG;
     if (max_rows == 0 || n_docs == 0) return HPD_OK;
-    const bool order = ord.active_slot != nullptr;
-    if (!q || !suffix_k || !suffix_v || !doc_kv_start || !doc_prefix_len || !doc_active_start || !doc_id ||
-        !n_active || !o || !workspace) return HPD_E_ARG;
+    const bool order = ord.prefix_vis != nullptr;
+    const bool slots = ord.active_slot != nullptr;       // position-order mode with branch caches (not the prefill)
+    if (!q || !doc_kv_start || !doc_prefix_len || !doc_active_start || !doc_id || !n_active || !o || !workspace) return HPD_E_ARG;
+    if ((!order || slots) && (!suffix_k || !suffix_v)) return HPD_E_ARG;
     if (!order && (!suffix_off || !suffix_len)) return HPD_E_ARG;
-    if (order && (!ord.doc_slot_start || !ord.slot_depth || !ord.slot_alive || !ord.prefix_vis)) return HPD_E_ARG;
+    if (slots && (!ord.doc_slot_start || !ord.slot_depth || !ord.slot_alive)) return HPD_E_ARG;
     if (total_prefix_tokens > 0 && (!prefix_k || !prefix_v)) return HPD_E_ARG;
     if (!aligned16(q) || !aligned16(prefix_k) || !aligned16(prefix_v) || !aligned16(suffix_k) ||
         !aligned16(suffix_v) || !aligned16(o) || !aligned16(workspace)) return HPD_E_ARG;
@@ -237,8 +238,9 @@ static int attn_common(const hpd_geom* geom, int n_docs, int max_rows, int n_slo
     a.q = static_cast<const __nv_bfloat16*>(q);
     a.prefix_k = static_cast<const __nv_bfloat16*>(prefix_k);
     a.prefix_v = static_cast<const __nv_bfloat16*>(prefix_v);
-    a.suffix_k = static_cast<const __nv_bfloat16*>(suffix_k);
-    a.suffix_v = static_cast<const __nv_bfloat16*>(suffix_v);
+    // without a branch cache (the prefill) the cache's tensor maps still need an address: the prefix tensors', never used
+    a.suffix_k = static_cast<const __nv_bfloat16*>(suffix_k ? suffix_k : prefix_k);
+    a.suffix_v = static_cast<const __nv_bfloat16*>(suffix_v ? suffix_v : prefix_v);
     a.doc_kv_start = doc_kv_start; a.doc_prefix_len = doc_prefix_len; a.doc_active_start = doc_active_start;
     a.doc_id = doc_id; a.suffix_off = suffix_off; a.suffix_len = suffix_len; a.n_active = n_active;
     a.suffix_extra = suffix_includes_new ? 1 : 0;
@@ -280,6 +282,41 @@ int hpd_attn_decode_posorder(const hpd_geom* geom, int n_docs, int max_rows, int
     return attn_common(geom, n_docs, max_rows, n_slots, total_prefix_tokens, q, prefix_k, prefix_v, suffix_k, suffix_v,
                        doc_kv_start, doc_prefix_len, doc_active_start, doc_id, nullptr, nullptr, ord,
                        n_active, suffix_includes_new, o, lse, workspace, workspace_bytes, dev_status, stream);
+}
+
+int hpd_prefill_meta(const hpd_geom* geom, int n_docs, int n_slots, int total_tokens,
+                     const int32_t* doc_prefix_len, const int32_t* doc_branch_cnt, const int32_t* slot_vis, int32_t pos_gap,
+                     int32_t* doc_kv_start, int32_t* doc_slot_start, int32_t* tok_doc, int32_t* tok_pos, int32_t* tok_vis,
+                     int32_t* n_tokens, void* workspace, size_t workspace_bytes, void* stream)
+{
+    int rc = geom_check(geom);
+    if (rc != HPD_OK) return rc;
+    if (n_docs < 0 || n_slots < 0 || total_tokens < 0 || pos_gap < 0) return HPD_E_ARG;
+    if (!doc_kv_start || !doc_slot_start || !n_tokens || !workspace || !aligned16(workspace)) return HPD_E_ARG;
+    if (n_docs > 0 && (!doc_prefix_len || !doc_branch_cnt)) return HPD_E_ARG;
+    if (n_slots > 0 && !slot_vis) return HPD_E_ARG;
+    if (total_tokens > 0 && (!tok_doc || !tok_pos || !tok_vis)) return HPD_E_ARG;
+    const int n_sm = sm_count();
+    const WsLayout lay = ws_layout(*geom, n_docs, total_tokens, n_sm);
+    if (workspace_bytes < lay.total) return HPD_E_WORKSPACE;
+    return launch_prefill_meta(*geom, n_docs, total_tokens, pos_gap, doc_prefix_len, doc_branch_cnt, slot_vis, doc_kv_start,
+                               doc_slot_start, tok_doc, tok_pos, tok_vis, n_tokens, workspace, lay, n_sm,
+                               static_cast<cudaStream_t>(stream));
+}
+
+int hpd_prefill_attn(const hpd_geom* geom, int n_docs, int total_tokens,
+                     const void* q, const void* prefix_k, const void* prefix_v,
+                     const int32_t* doc_kv_start, const int32_t* doc_prefix_len, const int32_t* tok_doc, const int32_t* tok_vis,
+                     const int32_t* n_tokens, void* o, float* lse,
+                     void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream)
+{
+    if (total_tokens > 0 && n_docs > 0 && !tok_vis) return HPD_E_ARG;
+    OrderTables ord{};
+    ord.prefix_vis = tok_vis;
+    // rows = tokens: a group's rows are its tokens (CSR of rows = doc_kv_start), no branch cache, max_slots = total_tokens
+    return attn_common(geom, n_docs, total_tokens, total_tokens, total_tokens, q, prefix_k, prefix_v, nullptr, nullptr,
+                       doc_kv_start, doc_prefix_len, doc_kv_start, tok_doc, nullptr, nullptr, ord, n_tokens, 0, o, lse,
+                       workspace, workspace_bytes, dev_status, stream);
 }
 
 static int std_splits(const hpd_geom* g, int max_rows, int max_seq_len)

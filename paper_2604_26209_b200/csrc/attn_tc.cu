@@ -370,7 +370,8 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         int das0 = p.a.doc_active_start[it0.doc], dks0 = p.a.doc_kv_start[it0.doc];
         // position-order mode: first slot of the group and of the next one
         int dss1 = 0, dse1 = 0, dss0 = 0, dse0 = 0;
-        if constexpr (ORDER) {
+        const bool have_slots = ORDER && p.a.slot_depth != nullptr;      // false: no branch cache at all (the prefill)
+        if (have_slots) {
             dss1 = p.a.doc_slot_start[it1.doc]; dse1 = p.a.doc_slot_start[it1.doc + 1];
             dss0 = p.a.doc_slot_start[it0.doc]; dse0 = p.a.doc_slot_start[it0.doc + 1];
         }
@@ -386,10 +387,10 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     rs[r] = -1; rp[r] = 0;
                     if (w < n_units && b < it.row_count) {
                         const int row = das + it.row_begin + b;
-                        rs[r] = p.a.active_slot[row];
+                        rs[r] = have_slots ? p.a.active_slot[row] : 0;
                         rp[r] = p.a.prefix_vis[row];
                     }
-                    if (w < n_units && it.with_suffix && b < dse - dss) {
+                    if (have_slots && w < n_units && it.with_suffix && b < dse - dss) {
                         rl[r] = p.a.slot_depth[dss + b];
                         ro[r] = p.a.slot_alive[dss + b];
                     }
@@ -411,7 +412,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             const WorkItem it3 = item_of(w3);
             const int das2 = p.a.doc_active_start[it2.doc], dks2 = p.a.doc_kv_start[it2.doc];
             int dss2 = 0, dse2 = 0;
-            if constexpr (ORDER) { dss2 = p.a.doc_slot_start[it2.doc]; dse2 = p.a.doc_slot_start[it2.doc + 1]; }
+            if (have_slots) { dss2 = p.a.doc_slot_start[it2.doc]; dse2 = p.a.doc_slot_start[it2.doc + 1]; }
             int rl1[kRounds], ro1[kRounds], rs1[ORDER ? kRounds : 1], rp1[ORDER ? kRounds : 1];
             load_tab(w1, it1, das1, dss1, dse1, rl1, ro1, rs1, rp1);
             // ---- finish unit i: clamp, validate, scan, publish ----
@@ -430,12 +431,12 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     const int b = lane + 32 * r;
                     const int idx = (live && b < it0.row_count) ? rs0[r] - dss0 : -1;
                     if (b == it0.row_count - 1) last = idx;
-                    if (live && b < it0.row_count && (idx < 0 || idx >= kM || idx >= dse0 - dss0)) bad = 1;   // group too large or bad table
+                    if (have_slots && live && b < it0.row_count && (idx < 0 || idx >= kM || idx >= dse0 - dss0)) bad = 1;   // group too large or bad table
                     d.ridx[b] = static_cast<uint16_t>(idx < 0 || idx >= kM ? 0 : idx);
                     d.pvis[b] = (live && b < it0.row_count) ? rp0[r] - it0.key_begin : 0;
                 }
                 last = __reduce_max_sync(0xffffffffu, last);
-                nbr = (live && it0.with_suffix && last < kM) ? last + 1 : 0;
+                nbr = (have_slots && live && it0.with_suffix && last < kM) ? last + 1 : 0;
             }
 #pragma unroll
             for (int r = 0; r < kRounds; ++r) {
@@ -989,7 +990,7 @@ int launch_d(const AttnArgs& a)
 int launch_attn_tc(const AttnArgs& a)
 {
     if (!(a.g.sm_scale > 0.f)) return HPD_E_GEOM;
-    if (a.active_slot) return a.g.D == 128 ? launch_d<128, true>(a) : launch_d<64, true>(a);
+    if (a.prefix_vis) return a.g.D == 128 ? launch_d<128, true>(a) : launch_d<64, true>(a);
     return a.g.D == 128 ? launch_d<128, false>(a) : launch_d<64, false>(a);
 }
 

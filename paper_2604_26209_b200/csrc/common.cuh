@@ -125,6 +125,10 @@ int launch_build_meta(const hpd_geom& g, int n_docs, int n_slots, const int32_t*
                       int32_t* suffix_off, int32_t* suffix_len, int32_t* n_active, void* workspace,
                       const WsLayout& lay, int n_sm, int32_t* dev_status, cudaStream_t stream,
                       const int32_t* slot_vis = nullptr, int32_t* prefix_vis = nullptr);
+int launch_prefill_meta(const hpd_geom& g, int n_docs, int total_tokens, int32_t pos_gap, const int32_t* doc_prefix_len,
+                        const int32_t* doc_branch_cnt, const int32_t* slot_vis, int32_t* doc_kv_start, int32_t* doc_slot_start,
+                        int32_t* tok_doc, int32_t* tok_pos, int32_t* tok_vis, int32_t* n_tokens, void* workspace,
+                        const WsLayout& lay, int n_sm, cudaStream_t stream);
 int launch_rope(const hpd_geom& g, int max_rows, const int32_t* n_active, const int32_t* pos_id,
                 __nv_bfloat16* q, __nv_bfloat16* k_new, cudaStream_t stream);
 int launch_kv_append(const hpd_geom& g, int max_rows, int n_slots, const int32_t* n_active, const int32_t* suffix_off,

@@ -431,7 +431,107 @@ meta_fused_kernel(int n_docs, int n_slots, int32_t suffix_cap, int32_t pos_gap, 
     plan_block<kFusedThreads>(n_docs, G, Hkv, n_sm, doc_prefix_len, doc_active_start, hdr, work, split, work_cap, part_cap);
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// First inference step (Sec. 4.3.2): the rows are the prompt tokens themselves.  One launch writes, per token, its
+// group, Algorithm 2's position ID (a gap of pos_gap behind every attribute key: t + pos_gap * #{slots whose key ends
+// before t}) and its causal bound t + 1; and the attention's work list: (group, block of 128/G tokens) against the
+// keys [0, end of the block) -- later keys are masked for every row of the block, so they are not visited at all.
+// ---------------------------------------------------------------------------------------------------------------
+constexpr int kPrefillDocs = 2048;
+constexpr int kPrefillThreads = 256;
+
+__global__ void __launch_bounds__(kPrefillThreads)
+prefill_meta_kernel(int n_docs, int G, int32_t pos_gap,
+                    const int32_t* __restrict__ doc_prefix_len, const int32_t* __restrict__ doc_branch_cnt,
+                    const int32_t* __restrict__ slot_vis,
+                    int32_t* __restrict__ doc_kv_start, int32_t* __restrict__ doc_slot_start,
+                    int32_t* __restrict__ tok_doc, int32_t* __restrict__ tok_pos, int32_t* __restrict__ tok_vis,
+                    int32_t* __restrict__ n_tokens, WsHeader* __restrict__ hdr, WorkItem* __restrict__ work,
+                    DocSplit* __restrict__ split, int work_cap, int part_cap)
+{
+    __shared__ int sm[kPrefillThreads / 32 + 1];
+    __shared__ int s_kv[kPrefillDocs + 1], s_slot[kPrefillDocs + 1], s_item[kPrefillDocs + 1];
+    const int rpb = kTileM / G;                      // tokens per row block
+    int run_kv = 0, run_sl = 0, run_it = 0;
+    for (int base = 0; base < n_docs; base += kPrefillThreads) {
+        const int d = base + threadIdx.x;
+        const int l = d < n_docs ? doc_prefix_len[d] : 0;
+        const int c = d < n_docs ? doc_branch_cnt[d] : 0;
+        const int it = (l + rpb - 1) / rpb;
+        int tl, tc, ti;
+        const int el = block_excl_scan<kPrefillThreads>(l, sm, tl);
+        const int ec = block_excl_scan<kPrefillThreads>(c, sm, tc);
+        const int ei = block_excl_scan<kPrefillThreads>(it, sm, ti);
+        if (d < n_docs) { s_kv[d] = run_kv + el; s_slot[d] = run_sl + ec; s_item[d] = run_it + ei; }
+        run_kv += tl; run_sl += tc; run_it += ti;
+    }
+    if (threadIdx.x == 0) { s_kv[n_docs] = run_kv; s_slot[n_docs] = run_sl; s_item[n_docs] = run_it; }
+    __syncthreads();
+    const int n_tok = run_kv, n_items = min(run_it, work_cap);
+    auto doc_of = [&](const int* start, int x) {      // last d with start[d] <= x (empty groups share a start and are skipped)
+        int lo = 0, hi = n_docs;
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (start[mid] <= x) lo = mid; else hi = mid;
+        }
+        return lo;
+    };
+    const int stride = gridDim.x * kPrefillThreads;
+    for (int x = blockIdx.x * kPrefillThreads + threadIdx.x; x < n_tok; x += stride) {
+        const int d = doc_of(s_kv, x);
+        const int t = x - s_kv[d];
+        int lo = s_slot[d], hi = s_slot[d + 1];       // slots of the group whose key ends before token t: slot_vis <= t
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (slot_vis[mid] <= t) lo = mid + 1; else hi = mid;
+        }
+        tok_doc[x] = d;
+        tok_pos[x] = t + pos_gap * (lo - s_slot[d]);
+        tok_vis[x] = t + 1;
+    }
+    for (int x = blockIdx.x * kPrefillThreads + threadIdx.x; x < n_items; x += stride) {
+        const int d = doc_of(s_item, x);
+        const int m = x - s_item[d];
+        const int L = s_kv[d + 1] - s_kv[d];
+        WorkItem it;
+        it.doc = d; it.key_begin = 0; it.key_count = min(L, (m + 1) * rpb);
+        it.part_base = -1; it.row_begin = m * rpb; it.row_count = min(rpb, L - m * rpb);
+        it.with_suffix = 0; it.pad = 0;
+        work[x] = it;
+    }
+    if (blockIdx.x == 0) {
+        for (int d = threadIdx.x; d <= n_docs; d += kPrefillThreads) {
+            doc_kv_start[d] = s_kv[d];
+            doc_slot_start[d] = s_slot[d];
+            if (d < n_docs) { split[d].part_base = -1; split[d].n_chunks = 1; }
+        }
+        if (threadIdx.x == 0) {
+            *n_tokens = n_tok;
+            hdr->n_work = n_items; hdr->chunk_tokens = 0; hdr->n_part_rows = 0; hdr->any_split = 0;
+            hdr->ticket = 0; hdr->finished = 0; hdr->work_cap = work_cap; hdr->part_cap = part_cap;
+        }
+    }
+}
+
 }  // namespace
+
+int launch_prefill_meta(const hpd_geom& g, int n_docs, int total_tokens, int32_t pos_gap, const int32_t* doc_prefix_len,
+                        const int32_t* doc_branch_cnt, const int32_t* slot_vis, int32_t* doc_kv_start, int32_t* doc_slot_start,
+                        int32_t* tok_doc, int32_t* tok_pos, int32_t* tok_vis, int32_t* n_tokens, void* workspace,
+                        const WsLayout& lay, int n_sm, cudaStream_t stream)
+{
+    if (n_docs > kPrefillDocs) return HPD_E_CAPACITY;
+    char* ws = static_cast<char*>(workspace);
+    int blocks = (total_tokens + kPrefillThreads - 1) / kPrefillThreads;
+    if (blocks < 1) blocks = 1;
+    if (blocks > 4 * n_sm) blocks = 4 * n_sm;
+    prefill_meta_kernel<<<blocks, kPrefillThreads, 0, stream>>>(
+        n_docs, g.Hq / g.Hkv, pos_gap, doc_prefix_len, doc_branch_cnt, slot_vis, doc_kv_start, doc_slot_start, tok_doc, tok_pos,
+        tok_vis, n_tokens, reinterpret_cast<WsHeader*>(ws), reinterpret_cast<WorkItem*>(ws + lay.off_work),
+        reinterpret_cast<DocSplit*>(ws + lay.off_split), lay.work_cap, lay.part_cap);
+    HPD_CUDA_TRY(cudaGetLastError());
+    return HPD_OK;
+}
 
 WsLayout ws_layout(const hpd_geom& g, int max_docs, int max_slots, int n_sm)
 {
