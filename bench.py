@@ -517,6 +517,71 @@ def run_shared3(args):
     }), flush=True)
 
 
+def run_prefill(args):
+    """First inference step (Sec. 4.3.2): causal attention of every prompt token of P prompts (2048 prompt tokens + the
+    skeleton of 96 attribute keys each) with Algorithm 2's position IDs.  A step = hpd_rope over all prompt tokens (keys
+    rotated in place in the prefix cache) + hpd_prefill_attn; the tables are built once.  Compute-bound: the roofline is
+    the measured dense bf16 rate."""
+    import torch
+    from paper_2604_26209_b200 import binding as B
+    torch.cuda.set_device(0)
+    B.load()
+    P = int(args.workload.split("_p")[1])
+    s = _posorder_structure(P, 0)
+    s.name = f"prefill_p{P}"
+    g, dev, T = s.geom, "cuda", s.total_prefix
+    gen = torch.Generator(device=dev); gen.manual_seed(0)
+    rnd = lambda *shape: torch.randn(*shape, device=dev, dtype=torch.float32, generator=gen).to(torch.bfloat16)
+    q0, k0, pv = rnd(T, g.Hq, g.D), rnd(T, g.Hkv, g.D), rnd(T, g.Hkv, g.D)
+    q, pk = q0.clone(), k0.clone()
+    o = torch.zeros_like(q)
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    L, cnt, vis = i32(s.doc_prefix_len), i32(s.doc_branch_cnt), i32(s.slot_vis)
+    t = B.PrefillTables.alloc(g, s.n_docs, T, dev)
+    B.hpd_prefill_meta(g, s.n_docs, s.n_slots, T, L, cnt, vis, s.pos_gap, t)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        B.hpd_rope(g, T, t.n_tokens, t.tok_pos, q, pk)          # (rotating again and again changes values, not the work)
+        B.hpd_prefill_attn(g, s.n_docs, T, q, pk, pv, L, t, o, None)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0); sampler.start(); time.sleep(0.2)
+    K = max(1, min(args.steps, 5))
+    blocks, att, t_w0 = [], [], time.time()
+    while sum(blocks) < args.min_ms or len(blocks) < 3:
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * K + 1)]
+        torch.cuda.synchronize()
+        ev[0].record(stream)
+        for i in range(K):
+            B.hpd_rope(g, T, t.n_tokens, t.tok_pos, q, pk); ev[2 * i + 1].record(stream)
+            B.hpd_prefill_attn(g, s.n_docs, T, q, pk, pv, L, t, o, None); ev[2 * i + 2].record(stream)
+        torch.cuda.synchronize()
+        blocks.append(ev[0].elapsed_time(ev[2 * K]))
+        att.append(float(np.mean([ev[2 * i + 1].elapsed_time(ev[2 * i + 2]) for i in range(K)])))
+    sampler.window(t_w0, time.time())
+    Ld = s.doc_prefix_len.astype(np.int64)
+    flops = 4 * g.D * g.Hq * int((Ld * (Ld + 1) // 2).sum())          # causal: token t sees t + 1 keys
+    hs = block_stats(blocks)
+    ms_att = float(np.median(att))
+    peaks = measured_peaks()
+    tf = flops / (ms_att * 1e-3) / 1e12
+    print(json.dumps({
+        "metric": "prompt_tokens_per_s_first_inference_step", "value": T * K / (hs["median_ms"] * 1e-3), "unit": "prompt-tokens/s",
+        "n_gpus": 1, "steps": K, "warmup": args.warmup, "ms_per_step": hs["median_ms"] / K, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": s.name, "prompts": P, "tokens": T, "tokens_per_prompt": int(Ld.mean()), "geometry": "Hq32/Hkv8/D128",
+                   "launch": "direct calls (rope, attention)"},
+        "timing": {"headline": hs}, "clocks": sampler.stop(), "gpu_launches": 3 * K,
+        "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
+                     "traffic": None, "kernel": "hpd_prefill_attn", "ms_per_launch": ms_att, "algorithmic_flops": flops,
+                     "peak_source": peaks["source"]},
+        "dev_status": int(t.dev_status.item()),
+    }), flush=True)
+
+
 def spawn_ranks(args) -> int:
     """``--gpus N`` without a rank environment: start one process per GPU (the environment torchrun would give them),
     wait for all, pass rank 0's JSON line through."""
@@ -649,6 +714,8 @@ def main():
         run_loop(args)
     elif args.workload.startswith("shared3_p") and args.impl != "reference":
         run_shared3(args)
+    elif args.workload.startswith("prefill_p") and args.impl != "reference":
+        run_prefill(args)
     elif args.impl == "reference":
         run_reference(args)
     elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
