@@ -508,12 +508,13 @@ def run_shared3(args):
     torch.cuda.synchronize()
     n = sb.db.tables()["n_active"]
     sb.db.set_step_inputs(tb["q"][:n], tb["k_new"][:n], tb["v_new"][:n])
+    s.name += "_two_pass" if args.two_pass else ""
     for _ in range(args.warmup):
-        sb.step()
+        sb.step(args.two_pass)
     g = torch.cuda.CUDAGraph()
     torch.cuda.synchronize()
     with torch.cuda.graph(g):
-        sb.step()
+        sb.step(args.two_pass)
     stream = torch.cuda.current_stream()
     sampler = ClockSampler(0); sampler.start(); time.sleep(0.2)
     blocks, t_w0 = [], time.time()
@@ -531,11 +532,11 @@ def run_shared3(args):
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
     att = []
     for _ in range(20):
-        ev[0].record(stream); sb.attn(); ev[1].record(stream); torch.cuda.synchronize()
+        ev[0].record(stream); (sb.attn_two_pass() if args.two_pass else sb.attn()); ev[1].record(stream); torch.cuda.synchronize()
         att.append(ev[0].elapsed_time(ev[1]))
     ab = algorithmic_bytes(s)
     row = s.geom.Hkv * s.geom.D * 4
-    bytes_attn = ab["attn"] + LB * row + 2 * ab["qo"]            # + the block once, + the second result written and both read by the merge
+    bytes_attn = ab["attn"] + LB * row + (2 * ab["qo"] if args.two_pass else 0)   # + the block once (+ the merge pass's traffic)
     hs = block_stats(blocks)
     peaks = measured_peaks()
     ms_att = float(np.median(att))
@@ -545,10 +546,10 @@ def run_shared3(args):
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": s.name, "block_tokens": LB, "doc_tokens": 512 - LB, "prompts": P, "n_active": n,
                    "launch": "cuda graph replay of the step"},
-        "timing": {"headline": hs}, "clocks": sampler.stop(), "gpu_launches": 9 * args.steps,
+        "timing": {"headline": hs}, "clocks": sampler.stop(), "gpu_launches": (9 if args.two_pass else 4) * args.steps,
         "roofline": {"bound": "hbm", "achieved": bytes_attn / (ms_att * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": bytes_attn / (ms_att * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
-                     "kernel": "hpd_attn_decode x2 + hpd_merge_lse", "ms_per_launch": ms_att, "algorithmic_bytes": int(bytes_attn)},
+                     "kernel": "hpd_attn_decode x2 + hpd_merge_lse" if args.two_pass else "hpd_attn_decode_shared", "ms_per_launch": ms_att, "algorithmic_bytes": int(bytes_attn)},
         "dev_status": sb.db.status(),
     }), flush=True)
 
@@ -741,6 +742,7 @@ def main():
     ap.add_argument("--unfused", action="store_true", help="hpd_rope and hpd_kv_append as two launches instead of hpd_rope_append")
     ap.add_argument("--min-ms", type=float, default=1000.0, help="device time to cover with timed K-step blocks")
     ap.add_argument("--block-tokens", type=int, default=128, help="shared3 workloads: tokens of the block common to all documents")
+    ap.add_argument("--two-pass", action="store_true", help="shared3 workloads: block attention as a second launch + hpd_merge_lse")
     ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--loop-prompts", type=int, default=64)
     args = ap.parse_args()

@@ -173,8 +173,29 @@ int hpd_advance(const hpd_geom* geom /*host*/, int max_rows, const int32_t* n_ac
                 int32_t* n_alive, void* stream);
 
 /*
- * hpd_merge_lse -- three sharing levels (Sec. 4.3.5: the instruction and the attribute definitions are
- * shared among all documents).  A block of tokens common to several documents is attended ONCE per block
+ * hpd_attn_decode_shared -- hpd_attn_decode with a third sharing level in the same launch (Sec. 4.3.5: the
+ * instruction and the attribute definitions are shared among all documents): document d is preceded by block
+ * doc_block[d], rows [block_kv_start[b], +block_len[b]) of block_k / block_v [total_block_tokens, Hkv, D] (dev),
+ * stored once however many documents follow it.  Every (document, kv head) unit visits its block's tiles and its
+ * document's tiles; the block's bytes come from HBM once and from L2 afterwards.  Results equal those of the
+ * block stored in front of every document.  doc_block [n_docs], block_kv_start and block_len [n_blocks] int32 dev.
+ * Position IDs must count the block: build the tables with hpd_build_meta_skeleton, slot_vis = block length + L_d,
+ * pos_gap = 0.  Everything else as hpd_attn_decode (with total_block_tokens = 0 it is that call).
+ */
+int hpd_attn_decode_shared(const hpd_geom* geom /*host*/, int n_docs, int max_rows, int n_slots, int total_prefix_tokens,
+                           const void* q, const void* prefix_k, const void* prefix_v,
+                           const void* suffix_k, const void* suffix_v,
+                           const void* block_k, const void* block_v, int total_block_tokens,
+                           const int32_t* doc_block, const int32_t* block_kv_start, const int32_t* block_len,
+                           const int32_t* doc_kv_start, const int32_t* doc_prefix_len, const int32_t* doc_active_start,
+                           const int32_t* doc_id, const int32_t* suffix_off, const int32_t* suffix_len,
+                           const int32_t* n_active, int suffix_includes_new,
+                           void* o, float* lse,
+                           void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream);
+
+/*
+ * hpd_merge_lse -- three sharing levels as separate passes (the building block for caches that hpd_attn_decode_shared
+ * does not cover, e.g. a block shared across calls).  A block of tokens common to several documents is attended ONCE per block
  * for all rows below it by a second hpd_attn_decode call whose "documents" are the blocks (tables from a
  * second hpd_build_meta over the blocks, its own workspace, an all-zero suffix_len table and
  * suffix_includes_new = 0, the block's K/V as prefix); this call combines the two results per (row, head):

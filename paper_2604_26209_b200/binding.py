@@ -18,7 +18,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libhpd.so")
 
 EXPORTS = ("hpd_strerror", "hpd_last_cuda_error", "hpd_workspace_bytes", "hpd_build_meta", "hpd_rope",
-           "hpd_kv_append", "hpd_rope_append", "hpd_attn_decode", "hpd_build_meta_skeleton", "hpd_attn_decode_posorder", "hpd_advance", "hpd_merge_lse", "hpd_prefill_meta", "hpd_prefill_attn", "std_workspace_bytes", "std_attn_decode",
+           "hpd_kv_append", "hpd_rope_append", "hpd_attn_decode", "hpd_build_meta_skeleton", "hpd_attn_decode_posorder", "hpd_advance", "hpd_merge_lse", "hpd_prefill_meta", "hpd_prefill_attn", "hpd_attn_decode_shared", "std_workspace_bytes", "std_attn_decode",
            "std_attn_decode_static_max_bytes", "std_attn_decode_static")
 
 HPD_S_OVERFLOW, HPD_S_BAD_TABLE, HPD_S_TIMEOUT = 1, 2, 4
@@ -65,6 +65,9 @@ def load() -> C.CDLL:
                                         [vp, C.c_size_t, vp]
         lib.hpd_prefill_attn.restype = C.c_int
         lib.hpd_prefill_attn.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int] + [vp] * 10 + [vp, C.c_size_t, vp, vp]
+        lib.hpd_attn_decode_shared.restype = C.c_int
+        lib.hpd_attn_decode_shared.argtypes = [C.POINTER(HpdGeom), C.c_int, C.c_int, C.c_int, C.c_int] + [vp] * 7 + [C.c_int] + \
+                                              [vp] * 10 + [C.c_int, vp, vp, vp, C.c_size_t, vp, vp]
         lib.hpd_merge_lse.restype = C.c_int
         lib.hpd_merge_lse.argtypes = [C.POINTER(HpdGeom), C.c_int] + [vp] * 8
         lib.hpd_advance.restype = C.c_int
@@ -220,6 +223,19 @@ def hpd_prefill_attn(geom, n_docs, total_tokens, q, prefix_k, prefix_v, doc_pref
                                  _ptr(t.doc_kv_start), _ptr(doc_prefix_len), _ptr(t.tok_doc), _ptr(t.tok_vis), _ptr(t.n_tokens),
                                  _ptr(o), _ptr(lse), _ptr(t.workspace), t.workspace.numel(), _ptr(t.dev_status), _stream())
     _check(rc, "hpd_prefill_attn")
+
+
+def hpd_attn_decode_shared(geom, n_docs, max_rows, n_slots, total_prefix_tokens, q, prefix_k, prefix_v, suffix_k, suffix_v,
+                           block_k, block_v, total_block_tokens, doc_block, block_kv_start, block_len,
+                           doc_prefix_len, m: MetaTables, suffix_includes_new, o, lse=None):
+    g = make_geom(geom)
+    rc = load().hpd_attn_decode_shared(C.byref(g), n_docs, max_rows, n_slots, total_prefix_tokens, _ptr(q), _ptr(prefix_k),
+                                       _ptr(prefix_v), _ptr(suffix_k), _ptr(suffix_v), _ptr(block_k), _ptr(block_v),
+                                       int(total_block_tokens), _ptr(doc_block), _ptr(block_kv_start), _ptr(block_len),
+                                       _ptr(m.doc_kv_start), _ptr(doc_prefix_len), _ptr(m.doc_active_start), _ptr(m.doc_id),
+                                       _ptr(m.suffix_off), _ptr(m.suffix_len), _ptr(m.n_active), int(bool(suffix_includes_new)),
+                                       _ptr(o), _ptr(lse), _ptr(m.workspace), m.workspace.numel(), _ptr(m.dev_status), _stream())
+    _check(rc, "hpd_attn_decode_shared")
 
 
 def hpd_merge_lse(geom, max_rows, n_active, o_a, lse_a, o_b, lse_b, o, lse=None):

@@ -203,6 +203,10 @@ int hpd_merge_lse(const hpd_geom* geom, int max_rows, const int32_t* n_active, c
 struct OrderTables {                 // extra tables of the position-order mode (all null in the branch-local mode)
     const int32_t *doc_slot_start, *active_slot, *slot_depth, *prefix_vis;
     const uint8_t* slot_alive;
+    // third sharing level (branch-local mode only; all null otherwise)
+    const void *block_k, *block_v;
+    const int32_t *doc_block, *block_kv_start, *block_len;
+    int total_block;
 };
 
 static int attn_common(const hpd_geom* geom, int n_docs, int max_rows, int n_slots, int total_prefix_tokens,
@@ -246,6 +250,9 @@ static int attn_common(const hpd_geom* geom, int n_docs, int max_rows, int n_slo
     a.suffix_extra = suffix_includes_new ? 1 : 0;
     a.doc_slot_start = ord.doc_slot_start; a.active_slot = ord.active_slot; a.slot_depth = ord.slot_depth;
     a.prefix_vis = ord.prefix_vis; a.slot_alive = ord.slot_alive;
+    a.block_k = static_cast<const __nv_bfloat16*>(ord.block_k); a.block_v = static_cast<const __nv_bfloat16*>(ord.block_v);
+    a.doc_block = ord.doc_block; a.block_kv_start = ord.block_kv_start; a.block_len = ord.block_len;
+    a.total_block = ord.total_block;
     a.o = static_cast<__nv_bfloat16*>(o);
     a.lse = lse;
     a.workspace = workspace; a.lay = lay; a.dev_status = dev_status;
@@ -264,6 +271,32 @@ int hpd_attn_decode(const hpd_geom* geom, int n_docs, int max_rows, int n_slots,
 {
     return attn_common(geom, n_docs, max_rows, n_slots, total_prefix_tokens, q, prefix_k, prefix_v, suffix_k, suffix_v,
                        doc_kv_start, doc_prefix_len, doc_active_start, doc_id, suffix_off, suffix_len, OrderTables{},
+                       n_active, suffix_includes_new, o, lse, workspace, workspace_bytes, dev_status, stream);
+}
+
+int hpd_attn_decode_shared(const hpd_geom* geom, int n_docs, int max_rows, int n_slots, int total_prefix_tokens,
+                           const void* q, const void* prefix_k, const void* prefix_v,
+                           const void* suffix_k, const void* suffix_v,
+                           const void* block_k, const void* block_v, int total_block_tokens,
+                           const int32_t* doc_block, const int32_t* block_kv_start, const int32_t* block_len,
+                           const int32_t* doc_kv_start, const int32_t* doc_prefix_len, const int32_t* doc_active_start,
+                           const int32_t* doc_id, const int32_t* suffix_off, const int32_t* suffix_len,
+                           const int32_t* n_active, int suffix_includes_new,
+                           void* o, float* lse,
+                           void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream)
+{
+    if (total_block_tokens < 0) return HPD_E_ARG;
+    if (total_block_tokens == 0)                         // no block at all: the plain call
+        return hpd_attn_decode(geom, n_docs, max_rows, n_slots, total_prefix_tokens, q, prefix_k, prefix_v, suffix_k, suffix_v,
+                               doc_kv_start, doc_prefix_len, doc_active_start, doc_id, suffix_off, suffix_len, n_active,
+                               suffix_includes_new, o, lse, workspace, workspace_bytes, dev_status, stream);
+    if (!block_k || !block_v || !doc_block || !block_kv_start || !block_len || !aligned16(block_k) || !aligned16(block_v))
+        return HPD_E_ARG;
+    OrderTables ord{};
+    ord.block_k = block_k; ord.block_v = block_v; ord.doc_block = doc_block; ord.block_kv_start = block_kv_start;
+    ord.block_len = block_len; ord.total_block = total_block_tokens;
+    return attn_common(geom, n_docs, max_rows, n_slots, total_prefix_tokens, q, prefix_k, prefix_v, suffix_k, suffix_v,
+                       doc_kv_start, doc_prefix_len, doc_active_start, doc_id, suffix_off, suffix_len, ord,
                        n_active, suffix_includes_new, o, lse, workspace, workspace_bytes, dev_status, stream);
 }
 

@@ -105,7 +105,8 @@ struct UnitDesc {
     int head, key_count, part_base, row_begin, nb /*branches*/;
     int row0;        // first global row
     int kv_row0;     // first global prefix token row
-    int pad[2];
+    int blk_count;   // tokens of the block shared by several documents that precede this unit's prefix chunk (0: none)
+    int blk_row0;    // first token row of that block in the block tensors
     uint16_t cs[kM];     // per branch: packed column of its first cached token
     uint16_t len[kM];    // per branch: cached tokens visible (0 for a bad table entry)
     // position-order mode: the branches above are ALL slots of the group up to the unit's last row (live or retired);
@@ -227,13 +228,14 @@ __device__ __forceinline__ uint32_t make_idesc(int N, int b_mn_major) {
 // per-unit bookkeeping
 // ------------------------------------------------------------------------------------------------
 struct Unit {        // the scalars of a descriptor, in registers
-    int nt, np, stot, head, key_count, part_base, row_begin, nb, row0, kv_row0;
+    int nt, np, stot, head, key_count, part_base, row_begin, nb, row0, kv_row0, blk_count, blk_row0;
 };
 
 __device__ __forceinline__ Unit read_unit(const UnitDesc& d) {
     Unit u;
     u.nt = d.nt; u.np = d.np; u.stot = d.stot; u.head = d.head; u.key_count = d.key_count; u.part_base = d.part_base;
     u.row_begin = d.row_begin; u.nb = d.nb; u.row0 = d.row0; u.kv_row0 = d.kv_row0;
+    u.blk_count = d.blk_count; u.blk_row0 = d.blk_row0;
     return u;
 }
 
@@ -241,17 +243,25 @@ __device__ __forceinline__ Unit read_unit(const UnitDesc& d) {
 // branch (and half), every lane placing the part of its branches that falls into the tile.  Boxes have the exact height
 // of the piece (tensor maps for 1..16 rows), so nothing beyond a branch's length is ever read: whatever lies there in
 // the cache -- possibly NaN -- must not meet a zero probability, and the packing needs no padding.
+// Tile order of a unit: the suffix tiles, the tiles of the shared block (if any), the tiles of the document's prefix chunk.
+__device__ __forceinline__ int block_tiles(const Unit& u) { return (u.blk_count + kN - 1) / kN; }
+
 template <int D>
 __device__ __forceinline__ void fill_tile(const Unit& u, int t, const int (&cs)[kRounds], const int (&len)[kRounds], const int (&off)[kRounds],
-                                          int lane, uint8_t* tile, unsigned long long* full, const CUtensorMap* pre, const CUtensorMap* suf)
+                                          int lane, uint8_t* tile, unsigned long long* full, const CUtensorMap* pre, const CUtensorMap* blk,
+                                          const CUtensorMap* suf)
 {
     using C = Cfg<D>;
-    const int ns = u.nt - u.np;
+    const int nbt = block_tiles(u);
+    const int ns = u.nt - u.np - nbt;
     if (t >= ns) {
         if (lane == 0) {
             mbar_expect_tx(full, C::KV_BYTES);
+            const bool in_block = t - ns < nbt;
+            const CUtensorMap* m = in_block ? blk : pre;
+            const int row = in_block ? u.blk_row0 + (t - ns) * kN : u.kv_row0 + (t - ns - nbt) * kN;
             for (int h = 0; h < C::HALVES; ++h)
-                tma_load_3d(tile + h * kKHalf, pre, full, h * 64, u.head, u.kv_row0 + (t - ns) * kN);
+                tma_load_3d(tile + h * kKHalf, m, full, h * 64, u.head, row);
         }
     } else {
         const int c_lo = t * kN, c_hi = min(u.stot, c_lo + kN);
@@ -288,10 +298,14 @@ __device__ __forceinline__ void fill_tile(const Unit& u, int t, const int (&cs)[
 //                tokens of every slot of the group up to and including its own -- live or retired --, which is "position
 //                ID not larger than mine" under Algorithm 2's K_max gaps.  Branch tokens are packed back to back in slot
 //                order, so a row's visible packed columns are one range starting at 0.
-template <int D, bool ORDER>
+// BLOCK = true:  a third sharing level (Sec. 4.3.5): the documents' prefixes are preceded by a block of tokens common to
+//                several documents (instruction, attribute definitions), stored once in tensors of its own; a unit visits the
+//                block's tiles between its suffix tiles and its document's tiles.
+template <int D, bool ORDER, bool BLOCK>
 __global__ void __launch_bounds__(kThreads, 1)
 hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                   const __grid_constant__ CUtensorMap map_v, const __grid_constant__ SufMaps smaps, const TcParams p)
+                   const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_bk,
+                   const __grid_constant__ CUtensorMap map_bv, const __grid_constant__ SufMaps smaps, const TcParams p)
 {
     using C = Cfg<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -368,6 +382,13 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         WorkItem it2 = item_of(w2), it1 = item_of(w1), it0 = item_of(w0);
         int das1 = p.a.doc_active_start[it1.doc], dks1 = p.a.doc_kv_start[it1.doc];
         int das0 = p.a.doc_active_start[it0.doc], dks0 = p.a.doc_kv_start[it0.doc];
+        // shared block of the unit's document: its id one stage ahead of its first row and length
+        int blk1 = 0, bks0 = 0, bln0 = 0;
+        if constexpr (BLOCK) {
+            blk1 = p.a.doc_block[it1.doc];
+            const int blk0 = p.a.doc_block[it0.doc];
+            bks0 = p.a.block_kv_start[blk0]; bln0 = p.a.block_len[blk0];
+        }
         // position-order mode: first slot of the group and of the next one
         int dss1 = 0, dse1 = 0, dss0 = 0, dse0 = 0;
         const bool have_slots = ORDER && p.a.slot_depth != nullptr;      // false: no branch cache at all (the prefill)
@@ -415,6 +436,11 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             if (have_slots) { dss2 = p.a.doc_slot_start[it2.doc]; dse2 = p.a.doc_slot_start[it2.doc + 1]; }
             int rl1[kRounds], ro1[kRounds], rs1[ORDER ? kRounds : 1], rp1[ORDER ? kRounds : 1];
             load_tab(w1, it1, das1, dss1, dse1, rl1, ro1, rs1, rp1);
+            int blk2 = 0, bks1 = 0, bln1 = 0;
+            if constexpr (BLOCK) {
+                blk2 = p.a.doc_block[it2.doc];
+                bks1 = p.a.block_kv_start[blk1]; bln1 = p.a.block_len[blk1];
+            }
             // ---- finish unit i: clamp, validate, scan, publish ----
             if (ui >= 1) {                               // the pipeline's consumers have copied the previous descriptor
                 ok = mbar_wait_warp(&misc->desc_empty[x], (ui - 1) & 1, misc);
@@ -468,14 +494,17 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             }
             if (__any_sync(0xffffffffu, bad) && lane == 0 && p.a.dev_status) atomicOr(p.a.dev_status, HPD_S_BAD_TABLE);
             Unit u;
+            u.blk_count = (BLOCK && live && it0.key_begin == 0 && bln0 > 0) ? bln0 : 0;     // the block goes with the document's first chunk
+            u.blk_row0 = bks0;
             u.np = live ? (it0.key_count + kN - 1) / kN : 0;
-            u.nt = live ? u.np + (carry + kN - 1) / kN : -1;
+            u.nt = live ? u.np + block_tiles(u) + (carry + kN - 1) / kN : -1;
             u.stot = carry; u.head = w0 % Hkv; u.key_count = it0.key_count; u.part_base = it0.part_base;
             u.row_begin = it0.row_begin; u.nb = it0.row_count;
             u.row0 = das0 + it0.row_begin; u.kv_row0 = dks0 + it0.key_begin;
             if (lane == 0) {
                 d.nt = u.nt; d.np = u.np; d.stot = u.stot; d.head = u.head; d.key_count = u.key_count; d.part_base = u.part_base;
                 d.row_begin = u.row_begin; d.nb = u.nb; d.row0 = u.row0; d.kv_row0 = u.kv_row0;
+                d.blk_count = u.blk_count; d.blk_row0 = u.blk_row0;
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&misc->desc_full[x]);
@@ -487,7 +516,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     const int ks = kc % C::NK;
                     ok = mbar_wait_warp(&misc->k_empty[x][ks], ((kc / C::NK) & 1) ^ 1, misc);
                     if (!ok) break;
-                    fill_tile<D>(u, t, cs, len, off, lane, k_ring + ks * C::KV_BYTES, &misc->k_full[x][ks], &map_k, smaps.k);
+                    fill_tile<D>(u, t, cs, len, off, lane, k_ring + ks * C::KV_BYTES, &misc->k_full[x][ks], &map_k, &map_bk, smaps.k);
                     ++kc;
                     if (t == 0) {
                         // The Q tile is asked for after the unit's first K tile: its buffer is released late in the
@@ -506,7 +535,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     const int vs = vc % C::NV;
                     ok = mbar_wait_warp(&misc->v_empty[x][vs], ((vc / C::NV) & 1) ^ 1, misc);
                     if (!ok) break;
-                    fill_tile<D>(u, t - 1, cs, len, off, lane, v_ring + vs * C::KV_BYTES, &misc->v_full[x][vs], &map_v, smaps.v);
+                    fill_tile<D>(u, t - 1, cs, len, off, lane, v_ring + vs * C::KV_BYTES, &misc->v_full[x][vs], &map_v, &map_bv, smaps.v);
                     ++vc;
                 }
                 __syncwarp();
@@ -516,6 +545,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             it0 = it1; it1 = it2; it2 = it3;
             das0 = das1; dks0 = dks1; das1 = das2; dks1 = dks2;
             if constexpr (ORDER) { dss0 = dss1; dse0 = dse1; dss1 = dss2; dse1 = dse2; }
+            if constexpr (BLOCK) { bks0 = bks1; bln0 = bln1; blk1 = blk2; }
 #pragma unroll
             for (int r = 0; r < kRounds; ++r) {
                 rl0[r] = rl1[r]; ro0[r] = ro1[r];
@@ -544,10 +574,18 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 if (u.nt < 0) break;
                 const int nt = u.nt;
                 if (nt == 0) continue;
-                const int ns = nt - u.np;
-                // columns of tile j: only the last suffix tile and the last prefix tile can be partial
+                const int nbt = BLOCK ? block_tiles(u) : 0;
+                const int ns = nt - u.np - nbt;
+                // columns of tile j: only the last suffix tile, the last block tile and the last prefix tile can be partial
                 const int last_s = u.stot - (ns - 1) * kN, last_p = u.key_count - (u.np - 1) * kN;
-                auto cols16 = [&](int j) { return ((j == ns - 1 ? last_s : (j == nt - 1 ? last_p : kN)) + 15) >> 4; };
+                const int last_b = u.blk_count - (nbt - 1) * kN;
+                auto cols16 = [&](int j) {
+                    int c = kN;
+                    if (j == ns - 1) c = last_s;
+                    else if (BLOCK && nbt > 0 && j == ns + nbt - 1) c = last_b;
+                    else if (j == nt - 1 && u.np > 0) c = last_p;
+                    return (c + 15) >> 4;
+                };
                 ok = mbar_wait(&misc->q_full[x], qc & 1, misc);
                 ++qc;
                 auto issue_qk = [&](int j) {
@@ -643,9 +681,12 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 // none of them (known from the descriptor alone) skips the tile's scores and writes zero probabilities.
                 int lo = 0, hi = 0;
                 if (warp_active) {
-                    const int ns = nt - u.np;
-                    if (j >= ns) {
-                        hi = min(kN, (ORDER ? min(u.key_count, my_pv) : u.key_count) - (j - ns) * kN);
+                    const int nbt = BLOCK ? block_tiles(u) : 0;
+                    const int ns = nt - u.np - nbt;
+                    if (BLOCK && j >= ns && j < ns + nbt) {
+                        hi = min(kN, u.blk_count - (j - ns) * kN);
+                    } else if (j >= ns) {
+                        hi = min(kN, (ORDER ? min(u.key_count, my_pv) : u.key_count) - (j - ns - nbt) * kN);
                         if (hi < 0) hi = 0;
                     } else {
                         const int base = j * kN;
@@ -919,7 +960,7 @@ bool make_q_map(CUtensorMap* m, const void* base, int D, int G, int Hkv, long lo
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D, bool ORDER>
+template <int D, bool ORDER, bool BLOCK>
 int launch_d(const AttnArgs& a)
 {
     using C = Cfg<D>;
@@ -927,7 +968,7 @@ int launch_d(const AttnArgs& a)
     static std::atomic<bool> attr_set[kMaxDevices];
     const int dev = current_device();
     if (dev < 0 || dev >= kMaxDevices || !attr_set[dev].load(std::memory_order_acquire)) {
-        HPD_CUDA_TRY(cudaFuncSetAttribute(hpd_attn_tc_kernel<D, ORDER>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
+        HPD_CUDA_TRY(cudaFuncSetAttribute(hpd_attn_tc_kernel<D, ORDER, BLOCK>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
         if (dev >= 0 && dev < kMaxDevices) attr_set[dev].store(true, std::memory_order_release);
     }
     const int G = a.g.Hq / a.g.Hkv;
@@ -979,7 +1020,14 @@ int launch_d(const AttnArgs& a)
     p.scale_log2 = a.g.sm_scale * kLog2e;
     p.G = G;
     const int n_sm = sm_count();
-    hpd_attn_tc_kernel<D, ORDER><<<n_sm, kThreads, C::SMEM, a.stream>>>(mq, mk, mv, sm, p);
+    CUtensorMap mbk = mk, mbv = mv;                      // unused without a shared block
+    if constexpr (BLOCK) {
+        if (!make_kv_map(&mbk, a.block_k, D, a.g.Hkv, a.total_block, kN) || !make_kv_map(&mbv, a.block_v, D, a.g.Hkv, a.total_block, kN)) {
+            set_last_cuda_error(cudaErrorInvalidValue);
+            return HPD_E_CUDA;
+        }
+    }
+    hpd_attn_tc_kernel<D, ORDER, BLOCK><<<n_sm, kThreads, C::SMEM, a.stream>>>(mq, mk, mv, mbk, mbv, sm, p);
     hpd_merge_kernel<D><<<n_sm * 2, 256, 0, a.stream>>>(p, reinterpret_cast<const DocSplit*>(ws + a.lay.off_split));
     HPD_CUDA_TRY(cudaGetLastError());
     return HPD_OK;
@@ -990,8 +1038,9 @@ int launch_d(const AttnArgs& a)
 int launch_attn_tc(const AttnArgs& a)
 {
     if (!(a.g.sm_scale > 0.f)) return HPD_E_GEOM;
-    if (a.prefix_vis) return a.g.D == 128 ? launch_d<128, true>(a) : launch_d<64, true>(a);
-    return a.g.D == 128 ? launch_d<128, false>(a) : launch_d<64, false>(a);
+    if (a.prefix_vis) return a.g.D == 128 ? launch_d<128, true, false>(a) : launch_d<64, true, false>(a);
+    if (a.block_k) return a.g.D == 128 ? launch_d<128, false, true>(a) : launch_d<64, false, true>(a);
+    return a.g.D == 128 ? launch_d<128, false, false>(a) : launch_d<64, false, false>(a);
 }
 
 }  // namespace hpd

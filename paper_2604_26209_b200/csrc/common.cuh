@@ -95,6 +95,10 @@ struct AttnArgs {
     // position-order mode only (all null otherwise): slot tables of the groups and the rows' visible prefix lengths
     const int32_t *doc_slot_start, *active_slot, *slot_depth, *prefix_vis;
     const uint8_t* slot_alive;
+    // third sharing level only (all null otherwise): block K/V [total_block, Hkv, D], block of each document, blocks' rows
+    const __nv_bfloat16 *block_k, *block_v;
+    const int32_t *doc_block, *block_kv_start, *block_len;
+    int total_block;
     __nv_bfloat16* o;
     float* lse;
     void* workspace;

@@ -128,8 +128,8 @@ class DeviceBatch:
 
 class SharedBlockBatch:
     """Three sharing levels (Sec. 4.3.5): blocks of tokens common to several documents, the documents, the branches.
-    Two hpd_attn_decode calls -- rows against their document and branch cache, rows against their block -- and
-    hpd_merge_lse.  ``doc_block[d]`` = block of document d (blocks cover consecutive documents), ``block_len[b]`` tokens,
+    ``attn()`` is one hpd_attn_decode_shared launch; ``attn_two_pass()`` is the same result from two hpd_attn_decode
+    calls -- rows against their document and branch cache, rows against their block -- and hpd_merge_lse.  ``doc_block[d]`` = block of document d (blocks cover consecutive documents), ``block_len[b]`` tokens,
     ``block_k/v`` bf16 bits [sum block_len, Hkv, D]."""
 
     def __init__(self, s: Structure, t: Dict[str, np.ndarray], doc_block: np.ndarray, block_len: np.ndarray,
@@ -145,6 +145,8 @@ class SharedBlockBatch:
         cnt = np.zeros(self.n_blocks, np.int64)
         np.add.at(cnt, doc_block, s.doc_branch_cnt)
         self.block_len, self.block_cnt = i32(block_len), i32(cnt)
+        self.doc_block = i32(doc_block)
+        self.block_kv_start = i32(np.concatenate([[0], np.cumsum(block_len)])[:-1])
         self.total_block = int(np.sum(block_len))
         self.block_k = _bf16(block_k, device) if self.total_block else torch.zeros(8, dtype=torch.bfloat16, device=device)
         self.block_v = _bf16(block_v, device) if self.total_block else torch.zeros(8, dtype=torch.bfloat16, device=device)
@@ -160,17 +162,26 @@ class SharedBlockBatch:
         B.hpd_build_meta(self.db.g, self.n_blocks, s.n_slots, self.block_len, self.block_cnt, db.slot_depth, db.slot_alive, 0,
                          self.meta_b)
 
-    def attn(self):
+    def attn(self, lse=True):
+        db, s, g = self.db, self.db.s, self.db.g
+        B.hpd_attn_decode_shared(g, s.n_docs, s.n_slots, s.n_slots, s.total_prefix, db.q, db.prefix_k, db.prefix_v, db.suffix_k,
+                                 db.suffix_v, self.block_k, self.block_v, self.total_block, self.doc_block, self.block_kv_start,
+                                 self.block_len, db.doc_prefix_len, db.meta, True, db.o, db.lse if lse else None)
+
+    def attn_two_pass(self):
         db, s, g = self.db, self.db.s, self.db.g
         db.attn(True, lse=True)
         B.hpd_attn_decode(g, self.n_blocks, s.n_slots, s.n_slots, self.total_block, db.q, self.block_k, self.block_v,
                           db.suffix_k, db.suffix_v, self.block_len, self.meta_b_nosuffix, False, self.o_b, self.lse_b)
         B.hpd_merge_lse(g, s.n_slots, db.meta.n_active, db.o, db.lse, self.o_b, self.lse_b, db.o, db.lse)
 
-    def step(self):
-        self.build_meta()
+    def step(self, two_pass=False):
+        if two_pass:
+            self.build_meta()
+        else:
+            self.db.build_meta()
         self.db.rope_append()
-        self.attn()
+        self.attn_two_pass() if two_pass else self.attn()
 
 
 class DupBatch:

@@ -27,11 +27,20 @@ CASES = {
     "ragged": lambda: (synth.config_custom("b", Hq=8, Hkv=4, D=64, theta=10000.0, cap=6, prefix_lens=[90, 0, 140, 5, 70, 33],
                                            branch_cnts=[5, 3, 0, 40, 1, 7], depth_hi=6, seed=2, alive_frac=0.8),
                        [0, 0, 1, 1, 2, 2], [111, 0, 300]),
+    # few rows and long documents: the prefix is split over several work items, the block goes with the first chunk
+    "split_prefix": lambda: (synth.config_custom("c", Hq=32, Hkv=8, D=128, theta=500000.0, cap=8, prefix_lens=[3000, 2500],
+                                                 branch_cnts=[2, 1], depth_hi=8, seed=3),
+                             [0, 0], [200]),
+    # documents without a prefix of their own: the block is all they share
+    "block_only": lambda: (synth.config_custom("d", Hq=8, Hkv=2, D=128, theta=10000.0, cap=4, prefix_lens=[0, 0, 0],
+                                               branch_cnts=[9, 30, 2], depth_hi=4, seed=4),
+                           [0, 0, 1], [130, 64]),
 }
 
 
+@pytest.mark.parametrize("two_pass", [False, True], ids=["one_launch", "two_passes_and_merge"])
 @pytest.mark.parametrize("name", list(CASES))
-def test_shared_block_step_matches_oracle(name):
+def test_shared_block_step_matches_oracle(name, two_pass):
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
     from paper_2604_26209_b200 import runtime as rt
@@ -54,7 +63,7 @@ def test_shared_block_step_matches_oracle(name):
         assert np.array_equal(tabs[nm], getattr(meta, nm)), nm
     sb.db.set_step_inputs(tb["q"][act], tb["k_new"][act], tb["v_new"][act])
     sb.db.rope_append()
-    sb.attn()
+    sb.attn_two_pass() if two_pass else sb.attn()
     torch.cuda.synchronize()
     assert sb.db.status() == 0
     o = synth.bf16_bits_to_f32(rt.bits_of(sb.db.o))[:n]
