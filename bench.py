@@ -449,7 +449,7 @@ def run_ours(args):
         tp = os.path.join(ROOT, "profiles", "traffic.json")
         if os.path.exists(tp):
             traffic = json.load(open(tp)).get(f"hpd_attn_decode:{s.name}")
-        launches_per_step = 3 + (2 if args.unfused else 1) + 2      # table kernels, rope/append, attention + merge
+        launches_per_step = 1 + (2 if args.unfused else 1) + 2      # table kernel, rope/append, attention + merge
         n_steps_timed = K * (len(head_blocks) + len(ms_total_blocks) + len(e2e_blocks))
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
