@@ -248,8 +248,8 @@ __device__ __forceinline__ int block_tiles(const Unit& u) { return (u.blk_count 
 
 template <int D>
 __device__ __forceinline__ void fill_tile(const Unit& u, int t, const int (&cs)[kRounds], const int (&len)[kRounds], const int (&off)[kRounds],
-                                          int lane, uint8_t* tile, unsigned long long* full, const CUtensorMap* pre, const CUtensorMap* blk,
-                                          const CUtensorMap* suf)
+                                          int nrounds, int lane, uint8_t* tile, unsigned long long* full, const CUtensorMap* pre,
+                                          const CUtensorMap* blk, const CUtensorMap* suf)
 {
     using C = Cfg<D>;
     const int nbt = block_tiles(u);
@@ -264,16 +264,13 @@ __device__ __forceinline__ void fill_tile(const Unit& u, int t, const int (&cs)[
                 tma_load_3d(tile + h * kKHalf, m, full, h * 64, u.head, row);
         }
     } else {
+        // the packing has no gaps: every column of [c_lo, c_hi) is some branch's cached token, so the tile receives
+        // exactly c_hi - c_lo rows
         const int c_lo = t * kN, c_hi = min(u.stot, c_lo + kN);
-        int rows_mine = 0;
+        if (lane == 0) mbar_expect_tx(full, static_cast<uint32_t>(c_hi - c_lo) * D * 2);
 #pragma unroll
         for (int r = 0; r < kRounds; ++r) {
-            rows_mine += max(0, min(cs[r] + len[r], c_hi) - max(cs[r], c_lo));
-        }
-        const int rows_all = __reduce_add_sync(0xffffffffu, rows_mine);
-        if (lane == 0) mbar_expect_tx(full, static_cast<uint32_t>(rows_all) * D * 2);
-#pragma unroll
-        for (int r = 0; r < kRounds; ++r) {
+            if (r >= nrounds) break;                     // rounds of 32 branches beyond the unit's last branch
             const int lo = max(cs[r], c_lo), hi = min(cs[r] + len[r], c_hi);
             int n = hi - lo;
             int row = off[r] + (lo - cs[r]);
@@ -493,6 +490,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 carry += __shfl_sync(0xffffffffu, incl, 31);
             }
             if (__any_sync(0xffffffffu, bad) && lane == 0 && p.a.dev_status) atomicOr(p.a.dev_status, HPD_S_BAD_TABLE);
+            const int nrounds = ((ORDER ? nbr : ((live && it0.with_suffix) ? it0.row_count : 0)) + 31) >> 5;
             Unit u;
             u.blk_count = (BLOCK && live && it0.key_begin == 0 && bln0 > 0) ? bln0 : 0;     // the block goes with the document's first chunk
             u.blk_row0 = bks0;
@@ -516,7 +514,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     const int ks = kc % C::NK;
                     ok = mbar_wait_warp(&misc->k_empty[x][ks], ((kc / C::NK) & 1) ^ 1, misc);
                     if (!ok) break;
-                    fill_tile<D>(u, t, cs, len, off, lane, k_ring + ks * C::KV_BYTES, &misc->k_full[x][ks], &map_k, &map_bk, smaps.k);
+                    fill_tile<D>(u, t, cs, len, off, nrounds, lane, k_ring + ks * C::KV_BYTES, &misc->k_full[x][ks], &map_k, &map_bk, smaps.k);
                     ++kc;
                     if (t == 0) {
                         // The Q tile is asked for after the unit's first K tile: its buffer is released late in the
@@ -535,7 +533,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     const int vs = vc % C::NV;
                     ok = mbar_wait_warp(&misc->v_empty[x][vs], ((vc / C::NV) & 1) ^ 1, misc);
                     if (!ok) break;
-                    fill_tile<D>(u, t - 1, cs, len, off, lane, v_ring + vs * C::KV_BYTES, &misc->v_full[x][vs], &map_v, &map_bv, smaps.v);
+                    fill_tile<D>(u, t - 1, cs, len, off, nrounds, lane, v_ring + vs * C::KV_BYTES, &misc->v_full[x][vs], &map_v, &map_bv, smaps.v);
                     ++vc;
                 }
                 __syncwarp();
