@@ -45,6 +45,38 @@ __device__ __forceinline__ int block_excl_scan(int v, int* smem /* THREADS/32 + 
     return res;
 }
 
+// Two block-wide exclusive scans at the price of one: both values (and both totals) are below 2^31, so they share one
+// 64-bit word without carrying into each other.
+template <int THREADS>
+__device__ __forceinline__ void block_excl_scan2(int a, int b, long long* smem /* THREADS/32 + 1 */, int& ea, int& eb, int& ta, int& tb) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long v = static_cast<long long>(static_cast<unsigned>(a)) | (static_cast<long long>(b) << 32);
+    long long incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const long long t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) smem[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        const long long w = (lane < THREADS / 32) ? smem[lane] : 0;
+        long long wi = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const long long t = __shfl_up_sync(0xffffffffu, wi, o);
+            if (lane >= o) wi += t;
+        }
+        if (lane < THREADS / 32) smem[lane] = wi - w;
+        if (lane == 31) smem[THREADS / 32] = wi;
+    }
+    __syncthreads();
+    const long long res = incl - v + smem[warp], tot = smem[THREADS / 32];
+    __syncthreads();
+    ea = static_cast<int>(res & 0xffffffffll); eb = static_cast<int>(res >> 32);
+    ta = static_cast<int>(tot & 0xffffffffll); tb = static_cast<int>(tot >> 32);
+}
+
 __global__ void __launch_bounds__(kScanThreads)
 doc_scan_kernel(int n_docs, const int32_t* __restrict__ doc_prefix_len, const int32_t* __restrict__ doc_branch_cnt,
                 int32_t* __restrict__ doc_kv_start, int32_t* __restrict__ doc_slot_start)
@@ -173,11 +205,30 @@ __device__ __forceinline__ void plan_block(int n_docs, int G, int Hkv, int n_sm,
                                            int work_cap, int part_cap)
 {
     constexpr int kPlanThreads = THREADS;
-    __shared__ int sm[kPlanThreads / 32 + 1];
+    __shared__ long long sm2[kPlanThreads / 32 + 1];
     __shared__ long long red[kCand * 2];
     __shared__ int s_choice;
     const int rows_per_block = kTileM / G;
 
+    // the usual case first: whole documents already give one unit per SM or more -> nothing to weigh
+    if (threadIdx.x < kCand * 2) red[threadIdx.x] = 0;
+    __syncthreads();
+    {
+        long long whole = 0;
+        for (int d = threadIdx.x; d < n_docs; d += kPlanThreads) {
+            const int rows = __ldcg(doc_active_start + d + 1) - __ldcg(doc_active_start + d);
+            if (rows > 0) whole += (rows + rows_per_block - 1) / rows_per_block;
+        }
+        for (int o = 16; o > 0; o >>= 1) whole += __shfl_down_sync(0xffffffffu, whole, o);
+        if ((threadIdx.x & 31) == 0 && whole)
+            atomicAdd(reinterpret_cast<unsigned long long*>(&red[0]), static_cast<unsigned long long>(whole));
+    }
+    __syncthreads();
+    const bool enough = red[0] * Hkv >= n_sm;
+    __syncthreads();
+    if (enough) {
+        if (threadIdx.x == 0) s_choice = kCand - 1;
+    } else {
     if (threadIdx.x < kCand * 2) red[threadIdx.x] = 0;
     __syncthreads();
     {
@@ -219,6 +270,7 @@ __device__ __forceinline__ void plan_block(int n_docs, int G, int Hkv, int n_sm,
         }
         s_choice = c;
     }
+    }
     __syncthreads();
     const int cand = s_choice;
 
@@ -237,9 +289,9 @@ __device__ __forceinline__ void plan_block(int n_docs, int G, int Hkv, int n_sm,
         }
         const int my_items = ch * mb;
         const int my_part = ch > 1 ? ch * rows : 0;
-        int tot_i, tot_p;
-        const int ei = run_items + block_excl_scan<kPlanThreads>(my_items, sm, tot_i);
-        const int ep = run_part + block_excl_scan<kPlanThreads>(my_part, sm, tot_p);
+        int tot_i, tot_p, ei, ep;
+        block_excl_scan2<kPlanThreads>(my_items, my_part, sm2, ei, ep, tot_i, tot_p);
+        ei += run_items; ep += run_part;
         if (d < n_docs) {
             split[d].part_base = ch > 1 ? ep : -1;
             split[d].n_chunks = ch;
@@ -344,9 +396,15 @@ meta_fused_kernel(int n_docs, int n_slots, int32_t suffix_cap, int32_t pos_gap, 
                   int work_cap, int part_cap)
 {
     __shared__ int sm[kFusedThreads / 32 + 1];
+    __shared__ long long sm2[kFusedThreads / 32 + 1];
     __shared__ int s_slot_start[kFusedDocs + 1];
     __shared__ int s_last;
     const int first = blockIdx.x * kFusedThreads;
+    // this thread's slot: its flags are asked for now and used after the scans
+    const int s = first + threadIdx.x;
+    const int alive = (s < n_slots) && slot_alive[s] != 0;
+    const int depth = s < n_slots ? slot_depth[s] : 0;
+    const int my_vis = (slot_vis && s < n_slots) ? slot_vis[s] : 0;
 
     // ---- scans over documents: slot starts stay in shared memory, block 0 also publishes both scans ----
     {
@@ -355,9 +413,8 @@ meta_fused_kernel(int n_docs, int n_slots, int32_t suffix_cap, int32_t pos_gap, 
             const int d = base + threadIdx.x;
             const int l = d < n_docs ? doc_prefix_len[d] : 0;
             const int c = d < n_docs ? doc_branch_cnt[d] : 0;
-            int tot_l, tot_c;
-            const int el = block_excl_scan<kFusedThreads>(l, sm, tot_l);
-            const int ec = block_excl_scan<kFusedThreads>(c, sm, tot_c);
+            int tot_l, tot_c, el, ec;
+            block_excl_scan2<kFusedThreads>(l, c, sm2, el, ec, tot_l, tot_c);
             if (d < n_docs) {
                 s_slot_start[d] = run_sl + ec;
                 if (blockIdx.x == 0) { doc_kv_start[d] = run_kv + el; doc_slot_start[d] = run_sl + ec; }
@@ -373,14 +430,11 @@ meta_fused_kernel(int n_docs, int n_slots, int32_t suffix_cap, int32_t pos_gap, 
     // ---- live slots before this block and in total ----
     int before, total;
     {
-        int tot;
-        block_excl_scan<kFusedThreads>(count_alive(slot_alive, 0, min(first, n_slots)), sm, tot);
-        before = tot;
-        block_excl_scan<kFusedThreads>(count_alive(slot_alive, min(first, n_slots), n_slots), sm, tot);
-        total = before + tot;
+        int e0, e1, after;
+        block_excl_scan2<kFusedThreads>(count_alive(slot_alive, 0, min(first, n_slots)),
+                                        count_alive(slot_alive, min(first, n_slots), n_slots), sm2, e0, e1, before, after);
+        total = before + after;
     }
-    const int s = first + threadIdx.x;
-    const int alive = (s < n_slots) && slot_alive[s] != 0;
     int tot;
     const int excl = before + block_excl_scan<kFusedThreads>(alive, sm, tot);
 
@@ -398,8 +452,7 @@ meta_fused_kernel(int n_docs, int n_slots, int32_t suffix_cap, int32_t pos_gap, 
             for (int e = d - 1; e >= 0 && s_slot_start[e + 1] == s_slot_start[e]; --e) doc_active_start[e] = excl;
         }
         if (alive) {
-            const int depth = slot_depth[s];
-            const int anchor = slot_vis ? slot_vis[s] : doc_prefix_len[d];
+            const int anchor = slot_vis ? my_vis : doc_prefix_len[d];
             const int bs = anchor + j * pos_gap;
             active_slot[excl] = s;
             doc_id[excl] = d;
