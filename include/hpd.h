@@ -20,8 +20,12 @@
  *   - documents are numbered globally in prompt order; "slots" are all branches ever admitted,
  *     numbered globally and grouped by document; "rows" are the live slots of this step in
  *     ascending slot id.  G = Hq / Hkv.
- *   - call order of one step:  hpd_build_meta  (once per step)
- *                              per layer: hpd_rope -> hpd_kv_append -> hpd_attn_decode.
+ *   - call order of one step:  hpd_build_meta  (once per step; hpd_build_meta_skeleton in
+ *                                               position-order mode)
+ *                              per layer: hpd_rope_append  (or hpd_rope -> hpd_kv_append)
+ *                                         -> hpd_attn_decode  (or _shared / _posorder)
+ *                              hpd_advance  (once per step, after the last layer).
+ *     The first inference step over the prompt tokens is hpd_prefill_meta -> hpd_prefill_attn.
  */
 #ifndef HPD_H_
 #define HPD_H_
