@@ -197,17 +197,49 @@ __device__ __forceinline__ int chunks_of(int L, int cand) {
     return (L + S - 1) / S;
 }
 
-// The split-KV plan, run by ONE block of THREADS threads (doc_active_start must be complete and visible).
+// Longest units first.  The attention kernel hands units out in list order, a few per pipeline, so a long unit drawn
+// late leaves one pipeline running after the others have finished.  Lists of up to kSortItems items (from up to
+// kSortDocs documents) whose items differ in length are therefore written in descending order of an estimate of
+// their duration: one per prefix key, a constant per branch-cache column of the rows (the cached lengths are not
+// looked at: one pass over every row would cost more than it saves) and a constant per unit.  Ties keep document
+// order, so the list is reproducible.  Longer lists stay in document order: their units are short against the launch.
+constexpr int kSortItems = 2048;
+constexpr int kSortDocs = 2048;
+constexpr int kPlanScratchInts = kSortItems;                  // the sort keys
+constexpr uint32_t kCostMax = 0xFFFFFu;                       // 20 bits of cost above 12 bits of item index
+constexpr int kUnitCost = 2 * kTileN;                         // a unit's fixed part, in key columns
+constexpr int kBranchCost = 16;                               // per row and q head of the group: its cached tokens' columns
+
+template <int THREADS>
+__device__ __forceinline__ void sort_keys_ascending(uint32_t* key, int n2 /* power of two */)
+{
+    for (int k = 2; k <= n2; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int t = threadIdx.x; t < n2 / 2; t += THREADS) {
+                const int lo = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+                const int hi = lo + j;
+                const uint32_t a = key[lo], b = key[hi];
+                const bool up = (lo & k) == 0;
+                if ((a > b) == up) { key[lo] = b; key[hi] = a; }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+// The split-KV plan, run by ONE block of THREADS threads (doc_active_start must be complete and visible).  scratch: kPlanScratchInts ints of shared memory, rank: kSortItems entries.
 template <int THREADS>
 __device__ __forceinline__ void plan_block(int n_docs, int G, int Hkv, int n_sm,
                                            const int32_t* doc_prefix_len, const int32_t* doc_active_start,
+                                           int* scratch, uint16_t* rank,
                                            WsHeader* __restrict__ hdr, WorkItem* __restrict__ work, DocSplit* __restrict__ split,
                                            int work_cap, int part_cap)
 {
     constexpr int kPlanThreads = THREADS;
     __shared__ long long sm2[kPlanThreads / 32 + 1];
+    __shared__ int sm1[kPlanThreads / 32 + 1];
     __shared__ long long red[kCand * 2];
-    __shared__ int s_choice;
+    __shared__ int s_choice, s_cost_min, s_cost_max;
     const int rows_per_block = kTileM / G;
 
     // the usual case first: whole documents already give one unit per SM or more -> nothing to weigh
@@ -274,7 +306,59 @@ __device__ __forceinline__ void plan_block(int n_docs, int G, int Hkv, int n_sm,
     __syncthreads();
     const int cand = s_choice;
 
-    // emit the work list in document order: exclusive scans of items and partial rows per document
+    // ---- order of the list: rank[item in document order] = its place, longest first ----
+    bool sorted = false;
+    if (n_docs <= kSortDocs) {
+        uint32_t* s_key = reinterpret_cast<uint32_t*>(scratch);
+        if (threadIdx.x == 0) { s_cost_min = 0x7fffffff; s_cost_max = 0; }
+        __syncthreads();
+        int n_items = 0;
+        int cmin = 0x7fffffff, cmax = 0;
+        for (int base = 0; base < n_docs; base += kPlanThreads) {
+            const int d = base + threadIdx.x;
+            int rows = 0, L = 0, mb = 0, ch = 0;
+            if (d < n_docs) {
+                rows = __ldcg(doc_active_start + d + 1) - __ldcg(doc_active_start + d);
+                L = doc_prefix_len[d];
+                if (rows > 0) { mb = (rows + rows_per_block - 1) / rows_per_block; ch = chunks_of(L, cand); }
+            }
+            int tot;
+            const int ei = n_items + block_excl_scan<kPlanThreads>(ch * mb, sm1, tot);
+            if (d < n_docs) {
+                const int S = (cand == kCand - 1) ? L : (kTileN << cand);
+                for (int c = 0, w = ei; c < ch; ++c) {
+                    const int kc = max(min(S, L - c * S), 0);
+                    for (int m = 0; m < mb; ++m, ++w) {
+                        const int nr = min(rows_per_block, rows - m * rows_per_block);
+                        const int cost = min(kUnitCost + min(kc, static_cast<int>(kCostMax)) + (c == ch - 1 ? nr * G * kBranchCost : 0), static_cast<int>(kCostMax));
+                        cmin = min(cmin, cost); cmax = max(cmax, cost);
+                        if (w < kSortItems) s_key[w] = ((kCostMax - static_cast<uint32_t>(cost)) << 12) | static_cast<uint32_t>(w);
+                    }
+                }
+            }
+            n_items += tot;
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            cmin = min(cmin, __shfl_xor_sync(0xffffffffu, cmin, o));
+            cmax = max(cmax, __shfl_xor_sync(0xffffffffu, cmax, o));
+        }
+        if ((threadIdx.x & 31) == 0) { atomicMin(&s_cost_min, cmin); atomicMax(&s_cost_max, cmax); }
+        __syncthreads();
+        // worth the sort only when the units differ: more than a quarter between the shortest and the longest
+        if (n_items > 1 && n_items <= kSortItems && (s_cost_max - s_cost_min) * 4 > s_cost_max) {
+            sorted = true;
+            int n2 = 2;
+            while (n2 < n_items) n2 <<= 1;
+            for (int w = n_items + threadIdx.x; w < n2; w += kPlanThreads) s_key[w] = 0xFFFFFFFFu;
+            __syncthreads();
+            sort_keys_ascending<kPlanThreads>(s_key, n2);
+            for (int i = threadIdx.x; i < n_items; i += kPlanThreads) rank[s_key[i] & 0xFFFu] = static_cast<uint16_t>(i);
+            __syncthreads();
+        }
+    }
+
+    // emit the work list: exclusive scans of items and partial rows per document give an item's place in document
+    // order, rank[] its place in the list
     int run_items = 0, run_part = 0, any_split = 0;
     for (int base = 0; base < n_docs; base += kPlanThreads) {
         const int d = base + threadIdx.x;
@@ -311,7 +395,7 @@ __device__ __forceinline__ void plan_block(int n_docs, int G, int Hkv, int n_sm,
                     it.part_base = ch > 1 ? ep + c * rows : -1;
                     it.with_suffix = (c == ch - 1);
                     it.pad = 0;
-                    work[w] = it;
+                    work[sorted ? static_cast<int>(rank[w]) : w] = it;
                 }
             }
         }
@@ -351,7 +435,10 @@ plan_kernel(int n_docs, int n_slots, int G, int Hkv, int n_sm,
         }
         return;
     }
-    plan_block<kPlanThreads>(n_docs, G, Hkv, n_sm, doc_prefix_len, doc_active_start, hdr, work, split, work_cap, part_cap);
+    __shared__ int s_scratch[kPlanScratchInts];
+    __shared__ uint16_t s_rank[kSortItems];
+    plan_block<kPlanThreads>(n_docs, G, Hkv, n_sm, doc_prefix_len, doc_active_start, s_scratch, s_rank,
+                             hdr, work, split, work_cap, part_cap);
 }
 
 // ---------------------------------------------------------------------------------------------------------------
@@ -481,7 +568,10 @@ meta_fused_kernel(int n_docs, int n_slots, int32_t suffix_cap, int32_t pos_gap, 
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    plan_block<kFusedThreads>(n_docs, G, Hkv, n_sm, doc_prefix_len, doc_active_start, hdr, work, split, work_cap, part_cap);
+    static_assert(kFusedDocs + 1 >= kPlanScratchInts, "the document scan's shared array doubles as the plan's scratch");
+    __shared__ uint16_t s_rank[kSortItems];
+    plan_block<kFusedThreads>(n_docs, G, Hkv, n_sm, doc_prefix_len, doc_active_start, s_slot_start, s_rank,
+                              hdr, work, split, work_cap, part_cap);
 }
 
 // ---------------------------------------------------------------------------------------------------------------
