@@ -29,6 +29,7 @@
 //
 // All waits are bounded: a wait that gives up raises HPD_S_TIMEOUT in the status word and the CTA
 // drains and exits (TMEM is released on every path).
+#include <algorithm>
 #include <atomic>
 
 #include "common.cuh"
@@ -880,7 +881,9 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     }
 }
 
-// Merge of the partial results of documents whose prefix was split over several work items.
+// Merge of the partial results of documents whose prefix was split over several work items.  One warp per (row, q
+// head); the chunks' partials are fetched four at a time so that their loads are in flight together (the kernel is a
+// chain of L2 round trips, not of bytes).
 template <int D>
 __global__ void __launch_bounds__(256)
 hpd_merge_kernel(TcParams p, const DocSplit* __restrict__ split)
@@ -892,28 +895,52 @@ hpd_merge_kernel(TcParams p, const DocSplit* __restrict__ split)
     const int Hq = p.a.g.Hq;
     const int64_t n_w = static_cast<int64_t>(*p.a.n_active) * Hq;
     constexpr int E = D / 32;
+    constexpr int kBatch = 4;
     for (int64_t w = static_cast<int64_t>(blockIdx.x) * 8 + (threadIdx.x >> 5); w < n_w; w += static_cast<int64_t>(gridDim.x) * 8) {
         const int r = static_cast<int>(w / Hq), h = static_cast<int>(w % Hq);
         const int d = p.a.doc_id[r];
         const DocSplit sp = split[d];
         if (sp.n_chunks <= 1) continue;
-        const int rows_d = p.a.doc_active_start[d + 1] - p.a.doc_active_start[d];
-        const int rl = r - p.a.doc_active_start[d];
+        const int das = p.a.doc_active_start[d];
+        const int rows_d = p.a.doc_active_start[d + 1] - das;
+        const int64_t pr0 = (static_cast<int64_t>(sp.part_base) + (r - das)) * Hq + h;      // chunk c: pr0 + c * step
+        const int64_t step = static_cast<int64_t>(rows_d) * Hq;
         float M = -INFINITY;
-        for (int c = 0; c < sp.n_chunks; ++c) {
-            const int64_t pr = (static_cast<int64_t>(sp.part_base) + static_cast<int64_t>(c) * rows_d + rl) * Hq + h;
-            M = fmaxf(M, p.part_ml[pr * 2]);
+        for (int c0 = 0; c0 < sp.n_chunks; c0 += kBatch) {
+            float m[kBatch];
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i)
+                m[i] = c0 + i < sp.n_chunks ? p.part_ml[(pr0 + (c0 + i) * step) * 2] : -INFINITY;
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) M = fmaxf(M, m[i]);
         }
         float L = 0.f, acc[E];
 #pragma unroll
         for (int e = 0; e < E; ++e) acc[e] = 0.f;
-        for (int c = 0; c < sp.n_chunks; ++c) {
-            const int64_t pr = (static_cast<int64_t>(sp.part_base) + static_cast<int64_t>(c) * rows_d + rl) * Hq + h;
-            const float mc = p.part_ml[pr * 2];
-            const float f = mc == -INFINITY ? 0.f : exp2f(mc - M);
-            L += f * p.part_ml[pr * 2 + 1];
+        for (int c0 = 0; c0 < sp.n_chunks; c0 += kBatch) {
+            float2 ml[kBatch];
+            float o[kBatch][E];
 #pragma unroll
-            for (int e = 0; e < E; ++e) acc[e] = fmaf(f, p.part_o[pr * D + lane * E + e], acc[e]);
+            for (int i = 0; i < kBatch; ++i) {
+                const bool in = c0 + i < sp.n_chunks;
+                const int64_t pr = pr0 + (in ? c0 + i : 0) * step;
+                ml[i] = in ? *reinterpret_cast<const float2*>(p.part_ml + pr * 2) : make_float2(-INFINITY, 0.f);
+                if constexpr (E == 4) {
+                    const float4 v = *reinterpret_cast<const float4*>(p.part_o + pr * D + lane * E);
+                    o[i][0] = v.x; o[i][1] = v.y; o[i][2] = v.z; o[i][3] = v.w;
+                } else {
+                    const float2 v = *reinterpret_cast<const float2*>(p.part_o + pr * D + lane * E);
+                    o[i][0] = v.x; o[i][1] = v.y;
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) {
+                if (c0 + i >= sp.n_chunks) continue;
+                const float f = ml[i].x == -INFINITY ? 0.f : exp2f(ml[i].x - M);
+                L += f * ml[i].y;
+#pragma unroll
+                for (int e = 0; e < E; ++e) acc[e] = fmaf(f, o[i][e], acc[e]);
+            }
         }
         const float inv = L > 0.f ? 1.f / L : 0.f;
         __nv_bfloat16* op = p.a.o + w * D + lane * E;
@@ -1030,7 +1057,10 @@ int launch_d(const AttnArgs& a)
         }
     }
     hpd_attn_tc_kernel<D, ORDER, BLOCK><<<n_sm, kThreads, C::SMEM, a.stream>>>(mq, mk, mv, mbk, mbv, sm, p);
-    hpd_merge_kernel<D><<<n_sm * 2, 256, 0, a.stream>>>(p, reinterpret_cast<const DocSplit*>(ws + a.lay.off_split));
+    // one warp per (row, q head) where the rows allow it, at most one resident wave
+    const long long merge_blocks = (static_cast<long long>(a.max_rows) * a.g.Hq + 7) / 8;
+    const int merge_grid = static_cast<int>(std::min<long long>(std::max<long long>(merge_blocks, 1), 8ll * n_sm));
+    hpd_merge_kernel<D><<<merge_grid, 256, 0, a.stream>>>(p, reinterpret_cast<const DocSplit*>(ws + a.lay.off_split));
     HPD_CUDA_TRY(cudaGetLastError());
     return HPD_OK;
 }
