@@ -80,7 +80,18 @@ STRUCTS = {
         depth_hi=4092, seed=26)),
     "long_small": lambda: synth.config_custom("long", Hq=32, Hkv=8, D=128, theta=500000.0, cap=32,
                                               prefix_lens=[4096, 1025, 3000], branch_cnts=[12, 12, 12], depth_hi=32, seed=8),
+    # work lists around the size up to which the plan orders them longest unit first (2048 items): documents of very
+    # different lengths, one or two branches each, every one alive so that each document is exactly one item
+    "sorted_list_1500": lambda: _varied_docs(1500, 27),
+    "sorted_list_2048": lambda: _varied_docs(2048, 28),
+    "unsorted_list_2049": lambda: _varied_docs(2049, 29),
 }
+
+
+def _varied_docs(n, seed):
+    lens = [(37 * i) % 331 + (900 if i % 97 == 0 else 0) for i in range(n)]
+    return synth.config_custom("varied", Hq=4, Hkv=1, D=64, theta=10000.0, cap=4, prefix_lens=lens,
+                               branch_cnts=[1 + (i % 2) for i in range(n)], depth_hi=4, seed=seed, alive_frac=1.0)
 
 
 def _run_step(rt, s, tb):
