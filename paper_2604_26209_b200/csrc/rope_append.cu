@@ -1,7 +1,7 @@
 // hpd_rope, hpd_kv_append and their fusion hpd_rope_append: the streaming kernels around the attention.
 //
-// All are pure HBM streaming (read + write of the step's new q/k/v rows); one CTA per row,
-// 16-byte accesses, grid sized by max_rows with an early exit on the device-side row count.
+// All are pure HBM streaming (read + write of the step's new q/k/v rows); one CTA per four rows (rotation) or per
+// row (append), 16-byte accesses, grid sized by max_rows with an early exit on the device-side row count.
 // The fused kernel rotates q and k in place, and while a rotated key chunk is still in registers also
 // stores it to the row's slot in the branch cache, then copies the value row there: one launch and one
 // read of k instead of two, the same bits as the two separate calls.
@@ -12,9 +12,11 @@ namespace hpd {
 namespace {
 
 constexpr int kRopeThreads = 256;
+constexpr int kRopeRows = 4;                         // rows per CTA: 4 x 64 angles give every thread one to evaluate
 
-// One CTA per row.  The row's D/2 (cos, sin) pairs are evaluated once, kept in shared memory as fp32 and applied to all
-// Hq + Hkv heads: each thread rotates 8 pairs at a time from one 16-byte load of the low half and one of the high half.
+// One CTA per four rows.  Every thread first asks for its share of the rows' q / k / v chunks (up to ten 16-byte loads in
+// flight per thread), then evaluates one of the rows' D/2 (cos, sin) pairs; they are kept in shared memory as fp32 and
+// applied to all Hq + Hkv heads: a thread rotates 8 pairs at a time from one 16-byte chunk of the low half and one of the high half.
 // Angles reach thousands of radians, where an fp32 product pos * inv_freq already loses ~1e-4 rad: the product and its
 // reduction to [-pi, pi] are taken in fp64 (inverse frequencies computed in fp64 on the host, 2*pi split in two doubles),
 // and only the reduced angle goes through the fp32 sine and cosine.
@@ -37,71 +39,134 @@ rope_kernel(int Hq, int Hkv, const InvFreq inv_freq, const int32_t* __restrict__
 {
     constexpr int HALF = D / 2;
     constexpr int CHUNKS = HALF / 8;                 // 16-byte chunks per half
-    __shared__ float cs[HALF], sn[HALF];
-    const int r = blockIdx.x;
-    if (r >= *n_active) return;
-    const int pos = pos_id[r];
-    // destination row in the branch cache (-1: slab full or table entry out of range -> status bit, no write)
-    int64_t dst_row = -1;
+    constexpr int R = kRopeRows;
+    constexpr int B = 5;                             // items a thread has in flight (the usual 32 + 8 heads of 128: all of them)
+    static_assert(R * HALF <= kRopeThreads, "one thread per angle of the CTA's rows");
+    __shared__ float cs[R][HALF], sn[R][HALF];
+    __shared__ long long s_dst[R];
+    const int r0 = blockIdx.x * R;
+    const int na = *n_active;
+    if (r0 >= na) return;
+    const int nr = min(R, na - r0);
+
+    // ---- every load that needs no angle is issued first: positions, slot tables, the first items of q / k / v ----
+    const int ar = threadIdx.x / HALF, ai = threadIdx.x % HALF;      // this thread's angle: row ar of the CTA, pair ai
+    const int pos = ar < nr ? pos_id[r0 + ar] : 0;
+    int t_len = 0;
+    int64_t t_off = 0;
     if constexpr (FUSED) {
-        const int len = ad.suffix_len[r];
-        const int64_t off = ad.suffix_off[r];
-        if (len >= ad.suffix_cap || len < 0) {
-            if (threadIdx.x == 0 && ad.dev_status) atomicOr(ad.dev_status, HPD_S_OVERFLOW);
-        } else if (off < 0 || off + len >= ad.cache_rows) {
-            if (threadIdx.x == 0 && ad.dev_status) atomicOr(ad.dev_status, HPD_S_BAD_TABLE);
-        } else {
-            dst_row = off + len;
+        if (threadIdx.x < nr) { t_len = ad.suffix_len[r0 + threadIdx.x]; t_off = ad.suffix_off[r0 + threadIdx.x]; }
+    }
+    const int items = (Hq + Hkv) * CHUNKS;           // 16-byte chunk pairs of one row
+    const int total = nr * items;
+    auto chunk_ptr = [&](int it, int& row, int& head, int& ch) -> uint4* {
+        row = it / items;
+        const int local = it - row * items;
+        head = local / CHUNKS; ch = local - head * CHUNKS;
+        __nv_bfloat16* base = head < Hq ? q + (static_cast<int64_t>(r0 + row) * Hq + head) * D
+                                        : k_new + (static_cast<int64_t>(r0 + row) * Hkv + (head - Hq)) * D;
+        return reinterpret_cast<uint4*>(base) + ch;
+    };
+    uint4 lo[B], hi[B];
+#pragma unroll
+    for (int k = 0; k < B; ++k) {
+        const int it = threadIdx.x + k * kRopeThreads;
+        if (it < total) {
+            int row, head, ch;
+            const uint4* pl = chunk_ptr(it, row, head, ch);
+            lo[k] = pl[0]; hi[k] = pl[CHUNKS];
         }
     }
-    if (threadIdx.x < HALF) {
-        const double ang = static_cast<double>(pos) * inv_freq.f[threadIdx.x];
+    // fused: the value rows' 16-byte pieces
+    const int row_u4 = Hkv * D / 8;
+    const int v_total = FUSED ? nr * row_u4 : 0;
+    uint4 vv[2];
+    if constexpr (FUSED) {
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const int it = threadIdx.x + k * kRopeThreads;
+            if (it < v_total) vv[k] = reinterpret_cast<const uint4*>(ad.v_new)[static_cast<int64_t>(r0) * row_u4 + it];
+        }
+    }
+
+    // ---- angles, and where each row goes in the branch cache (-1: slab full or table entry out of range -> status bit, no write) ----
+    if (ar < nr) {
+        const double ang = static_cast<double>(pos) * inv_freq.f[ai];
         const double k = rint(ang * 0.15915494309189535);                       // turns
         double r = fma(-k, 6.283185307179586, ang);                             // minus k * 2*pi (high part, then the rest)
         r = fma(-k, 2.4492935982947064e-16, r);
         float s, c;
         sincosf(static_cast<float>(r), &s, &c);
-        cs[threadIdx.x] = c;
-        sn[threadIdx.x] = s;
+        cs[ar][ai] = c;
+        sn[ar][ai] = s;
+    }
+    if constexpr (FUSED) {
+        if (threadIdx.x < nr) {
+            long long dst = -1;
+            if (t_len >= ad.suffix_cap || t_len < 0) {
+                if (ad.dev_status) atomicOr(ad.dev_status, HPD_S_OVERFLOW);
+            } else if (t_off < 0 || t_off + t_len >= ad.cache_rows) {
+                if (ad.dev_status) atomicOr(ad.dev_status, HPD_S_BAD_TABLE);
+            } else {
+                dst = t_off + t_len;
+            }
+            s_dst[threadIdx.x] = dst;
+        }
     }
     __syncthreads();
-    const int items = (Hq + Hkv) * CHUNKS;
-    // fused: the value row's 16-byte pieces are further items, so the threads left over by the rotation copy them
-    const int row_u4 = Hkv * D / 8;
-    const int all_items = (FUSED && dst_row >= 0) ? items + row_u4 : items;
-    for (int it = threadIdx.x; it < all_items; it += kRopeThreads) {
-        if constexpr (FUSED) {
-            if (it >= items) {
-                const int i = it - items;
-                reinterpret_cast<uint4*>(ad.suffix_v)[dst_row * row_u4 + i] =
-                    reinterpret_cast<const uint4*>(ad.v_new)[static_cast<int64_t>(r) * row_u4 + i];
-                continue;
+
+    // ---- rotate in place; the fused kernel also stores the rotated key chunks to the cache while they are in registers ----
+    for (int base = 0; base < total; base += B * kRopeThreads) {
+        if (base > 0) {
+#pragma unroll
+            for (int k = 0; k < B; ++k) {
+                const int it = base + threadIdx.x + k * kRopeThreads;
+                if (it < total) {
+                    int row, head, ch;
+                    const uint4* pl = chunk_ptr(it, row, head, ch);
+                    lo[k] = pl[0]; hi[k] = pl[CHUNKS];
+                }
             }
         }
-        const int head = it / CHUNKS, ch = it % CHUNKS;
-        __nv_bfloat16* base = head < Hq ? q + (static_cast<int64_t>(r) * Hq + head) * D
-                                        : k_new + (static_cast<int64_t>(r) * Hkv + (head - Hq)) * D;
-        uint4* plo = reinterpret_cast<uint4*>(base) + ch;
-        uint4* phi = reinterpret_cast<uint4*>(base + HALF) + ch;
-        uint4 lo = *plo, hi = *phi;
-        uint32_t* l = reinterpret_cast<uint32_t*>(&lo);
-        uint32_t* h = reinterpret_cast<uint32_t*>(&hi);
 #pragma unroll
-        for (int w = 0; w < 4; ++w) {
-            const int i = ch * 8 + w * 2;
-            const float a0 = bf16lo(l[w]), a1 = bf16hi(l[w]);
-            const float b0 = bf16lo(h[w]), b1 = bf16hi(h[w]);
-            const float c0 = cs[i], s0 = sn[i], c1 = cs[i + 1], s1 = sn[i + 1];
-            l[w] = pack_bf16(fmaf(a0, c0, -b0 * s0), fmaf(a1, c1, -b1 * s1));
-            h[w] = pack_bf16(fmaf(b0, c0, a0 * s0), fmaf(b1, c1, a1 * s1));
+        for (int k = 0; k < B; ++k) {
+            const int it = base + threadIdx.x + k * kRopeThreads;
+            if (it >= total) continue;
+            int row, head, ch;
+            uint4* pl = chunk_ptr(it, row, head, ch);
+            uint32_t* l = reinterpret_cast<uint32_t*>(&lo[k]);
+            uint32_t* h = reinterpret_cast<uint32_t*>(&hi[k]);
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+                const int i = ch * 8 + w * 2;
+                const float a0 = bf16lo(l[w]), a1 = bf16hi(l[w]);
+                const float b0 = bf16lo(h[w]), b1 = bf16hi(h[w]);
+                const float c0 = cs[row][i], s0 = sn[row][i], c1 = cs[row][i + 1], s1 = sn[row][i + 1];
+                l[w] = pack_bf16(fmaf(a0, c0, -b0 * s0), fmaf(a1, c1, -b1 * s1));
+                h[w] = pack_bf16(fmaf(b0, c0, a0 * s0), fmaf(b1, c1, a1 * s1));
+            }
+            pl[0] = lo[k];
+            pl[CHUNKS] = hi[k];
+            if constexpr (FUSED) {
+                const long long dst_row = s_dst[row];
+                if (head >= Hq && dst_row >= 0) {
+                    uint4* cd = reinterpret_cast<uint4*>(ad.suffix_k + (dst_row * Hkv + (head - Hq)) * D);
+                    cd[ch] = lo[k];
+                    cd[CHUNKS + ch] = hi[k];
+                }
+            }
         }
-        *plo = lo;
-        *phi = hi;
-        if constexpr (FUSED) {
-            if (head >= Hq && dst_row >= 0) {
-                uint4* cd = reinterpret_cast<uint4*>(ad.suffix_k + (dst_row * Hkv + (head - Hq)) * D);
-                cd[ch] = lo;
-                cd[CHUNKS + ch] = hi;
+    }
+    if constexpr (FUSED) {
+        for (int base = 0; base < v_total; base += 2 * kRopeThreads) {
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const int it = base + threadIdx.x + k * kRopeThreads;
+                if (it >= v_total) continue;
+                if (base > 0) vv[k] = reinterpret_cast<const uint4*>(ad.v_new)[static_cast<int64_t>(r0) * row_u4 + it];
+                const int row = it / row_u4;
+                const long long dst_row = s_dst[row];
+                if (dst_row >= 0) reinterpret_cast<uint4*>(ad.suffix_v)[dst_row * row_u4 + (it - row * row_u4)] = vv[k];
             }
         }
     }
@@ -234,9 +299,9 @@ int launch_rope(const hpd_geom& g, int max_rows, const int32_t* n_active, const 
     const InvFreq c = inv_freq_table(g);
     const AppendDst none{};
     if (g.D == 128)
-        rope_kernel<128, false><<<max_rows, kRopeThreads, 0, stream>>>(g.Hq, g.Hkv, c, n_active, pos_id, q, k_new, none);
+        rope_kernel<128, false><<<(max_rows + kRopeRows - 1) / kRopeRows, kRopeThreads, 0, stream>>>(g.Hq, g.Hkv, c, n_active, pos_id, q, k_new, none);
     else
-        rope_kernel<64, false><<<max_rows, kRopeThreads, 0, stream>>>(g.Hq, g.Hkv, c, n_active, pos_id, q, k_new, none);
+        rope_kernel<64, false><<<(max_rows + kRopeRows - 1) / kRopeRows, kRopeThreads, 0, stream>>>(g.Hq, g.Hkv, c, n_active, pos_id, q, k_new, none);
     HPD_CUDA_TRY(cudaGetLastError());
     return HPD_OK;
 }
@@ -251,9 +316,9 @@ int launch_rope_append(const hpd_geom& g, int max_rows, int n_slots, const int32
     const AppendDst ad{g.suffix_cap, static_cast<int64_t>(n_slots) * g.suffix_cap, suffix_off, suffix_len, v_new,
                        suffix_k, suffix_v, dev_status};
     if (g.D == 128)
-        rope_kernel<128, true><<<max_rows, kRopeThreads, 0, stream>>>(g.Hq, g.Hkv, c, n_active, pos_id, q, k_new, ad);
+        rope_kernel<128, true><<<(max_rows + kRopeRows - 1) / kRopeRows, kRopeThreads, 0, stream>>>(g.Hq, g.Hkv, c, n_active, pos_id, q, k_new, ad);
     else
-        rope_kernel<64, true><<<max_rows, kRopeThreads, 0, stream>>>(g.Hq, g.Hkv, c, n_active, pos_id, q, k_new, ad);
+        rope_kernel<64, true><<<(max_rows + kRopeRows - 1) / kRopeRows, kRopeThreads, 0, stream>>>(g.Hq, g.Hkv, c, n_active, pos_id, q, k_new, ad);
     HPD_CUDA_TRY(cudaGetLastError());
     return HPD_OK;
 }
