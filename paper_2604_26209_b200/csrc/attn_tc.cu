@@ -1057,9 +1057,11 @@ int launch_d(const AttnArgs& a)
         }
     }
     hpd_attn_tc_kernel<D, ORDER, BLOCK><<<n_sm, kThreads, C::SMEM, a.stream>>>(mq, mk, mv, mbk, mbv, sm, p);
-    // one warp per (row, q head) where the rows allow it, at most one resident wave
+    // one warp per (row, q head) where the rows allow it, at most one resident wave; with many documents nothing is
+    // split as a rule (the kernel then only rewinds the ticket counter) and a small grid is launched sooner
     const long long merge_blocks = (static_cast<long long>(a.max_rows) * a.g.Hq + 7) / 8;
-    const int merge_grid = static_cast<int>(std::min<long long>(std::max<long long>(merge_blocks, 1), 8ll * n_sm));
+    const long long merge_cap = static_cast<long long>(a.n_docs) * a.g.Hkv < 4ll * n_sm ? 8ll * n_sm : 2ll * n_sm;
+    const int merge_grid = static_cast<int>(std::min<long long>(std::max<long long>(merge_blocks, 1), merge_cap));
     hpd_merge_kernel<D><<<merge_grid, 256, 0, a.stream>>>(p, reinterpret_cast<const DocSplit*>(ws + a.lay.off_split));
     HPD_CUDA_TRY(cudaGetLastError());
     return HPD_OK;

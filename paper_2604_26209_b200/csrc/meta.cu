@@ -213,6 +213,11 @@ constexpr uint32_t kCostMax = 0xFFFFFu;                       // 20 bits of cost
 constexpr int kUnitCost = 2 * kTileN;                         // a unit's fixed part, in key columns
 constexpr int kBranchCost = 16;                               // per row and q head of the group: its cached tokens' columns
 
+// estimate of a unit's duration, in key columns: keys of the prefix chunk, rows whose branch caches the unit visits
+__device__ __forceinline__ int unit_cost(int keys, int branch_rows, int G) {
+    return min(kUnitCost + keys + branch_rows * G * kBranchCost, static_cast<int>(kCostMax));
+}
+
 template <int THREADS>
 __device__ __forceinline__ void sort_keys_ascending(uint32_t* key, int n2 /* power of two */)
 {
@@ -246,20 +251,38 @@ __device__ __forceinline__ void plan_block(int n_docs, int G, int Hkv, int n_sm,
     const int rows_per_block = kTileM / G;
 
     // the usual case first: whole documents already give one unit per SM or more -> nothing to weigh
+    // (the same pass weighs the whole documents' units: only lists whose units differ in length are put in order below)
     if (threadIdx.x < kCand * 2) red[threadIdx.x] = 0;
+    if (threadIdx.x == 0) { s_cost_min = 0x7fffffff; s_cost_max = 0; }
     __syncthreads();
     {
         long long whole = 0;
+        int cmin = 0x7fffffff, cmax = 0;
         for (int d = threadIdx.x; d < n_docs; d += kPlanThreads) {
             const int rows = __ldcg(doc_active_start + d + 1) - __ldcg(doc_active_start + d);
-            if (rows > 0) whole += (rows + rows_per_block - 1) / rows_per_block;
+            if (rows > 0) {
+                const int mb = (rows + rows_per_block - 1) / rows_per_block;
+                whole += mb;
+                const int L = min(max(doc_prefix_len[d], 0), static_cast<int>(kCostMax));
+                cmin = min(cmin, unit_cost(L, rows - (mb - 1) * rows_per_block, G));
+                cmax = max(cmax, unit_cost(L, min(rows, rows_per_block), G));
+            }
         }
-        for (int o = 16; o > 0; o >>= 1) whole += __shfl_down_sync(0xffffffffu, whole, o);
-        if ((threadIdx.x & 31) == 0 && whole)
+        for (int o = 16; o > 0; o >>= 1) {
+            whole += __shfl_down_sync(0xffffffffu, whole, o);
+            cmin = min(cmin, __shfl_xor_sync(0xffffffffu, cmin, o));
+            cmax = max(cmax, __shfl_xor_sync(0xffffffffu, cmax, o));
+        }
+        if ((threadIdx.x & 31) == 0 && whole) {
             atomicAdd(reinterpret_cast<unsigned long long*>(&red[0]), static_cast<unsigned long long>(whole));
+            atomicMin(&s_cost_min, cmin); atomicMax(&s_cost_max, cmax);
+        }
     }
     __syncthreads();
     const bool enough = red[0] * Hkv >= n_sm;
+    // worth the sort only when the units differ: more than a quarter between the shortest and the longest (a split
+    // list always goes through the pass below: its chunks differ)
+    const bool differ = !enough || (s_cost_max > s_cost_min && (s_cost_max - s_cost_min) * 4 > s_cost_max);
     __syncthreads();
     if (enough) {
         if (threadIdx.x == 0) s_choice = kCand - 1;
@@ -311,12 +334,9 @@ __device__ __forceinline__ void plan_block(int n_docs, int G, int Hkv, int n_sm,
 
     // ---- order of the list: rank[item in document order] = its place, longest first ----
     bool sorted = false;
-    if (n_docs <= kSortDocs) {
+    if (n_docs <= kSortDocs && differ) {
         uint32_t* s_key = reinterpret_cast<uint32_t*>(scratch);
-        if (threadIdx.x == 0) { s_cost_min = 0x7fffffff; s_cost_max = 0; }
-        __syncthreads();
         int n_items = 0;
-        int cmin = 0x7fffffff, cmax = 0;
         for (int base = 0; base < n_docs; base += kPlanThreads) {
             const int d = base + threadIdx.x;
             int rows = 0, L = 0, mb = 0, ch = 0;
@@ -333,22 +353,15 @@ __device__ __forceinline__ void plan_block(int n_docs, int G, int Hkv, int n_sm,
                     const int kc = max(min(S, L - c * S), 0);
                     for (int m = 0; m < mb; ++m, ++w) {
                         const int nr = min(rows_per_block, rows - m * rows_per_block);
-                        const int cost = min(kUnitCost + min(kc, static_cast<int>(kCostMax)) + (c == ch - 1 ? nr * G * kBranchCost : 0), static_cast<int>(kCostMax));
-                        cmin = min(cmin, cost); cmax = max(cmax, cost);
+                        const int cost = unit_cost(min(kc, static_cast<int>(kCostMax)), c == ch - 1 ? nr : 0, G);
                         if (w < kSortItems) s_key[w] = ((kCostMax - static_cast<uint32_t>(cost)) << 12) | static_cast<uint32_t>(w);
                     }
                 }
             }
             n_items += tot;
         }
-        for (int o = 16; o > 0; o >>= 1) {
-            cmin = min(cmin, __shfl_xor_sync(0xffffffffu, cmin, o));
-            cmax = max(cmax, __shfl_xor_sync(0xffffffffu, cmax, o));
-        }
-        if ((threadIdx.x & 31) == 0) { atomicMin(&s_cost_min, cmin); atomicMax(&s_cost_max, cmax); }
         __syncthreads();
-        // worth the sort only when the units differ: more than a quarter between the shortest and the longest
-        if (n_items > 1 && n_items <= kSortItems && (s_cost_max - s_cost_min) * 4 > s_cost_max) {
+        if (n_items > 1 && n_items <= kSortItems) {
             sorted = true;
             int n2 = 2;
             while (n2 < n_items) n2 <<= 1;
