@@ -361,12 +361,13 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         if (n_units == 0) {                              // nothing to do: publish the stop descriptor
             if (lane == 0) { d.nt = -1; mbar_arrive(&misc->desc_full[x]); }
         } else {
-        // The first units of a pipeline are fixed (round i hands unit i * 2 * grid + j to the j-th pipeline, j counted
-        // upwards in even rounds and downwards in odd ones: the list comes longest unit first, and the alternation
-        // keeps the pipelines' sums level), which fills the software pipeline without a chain of atomics and measured
+        // The first units of a pipeline are fixed (round i hands unit i * 2 * grid + j to the j-th pipeline; when the
+        // list comes longest unit first, j counts upwards in even rounds and downwards in odd ones, which keeps the
+        // pipelines' sums level), which fills the software pipeline without a chain of atomics and measured
         // slightly faster than drawing early; later units are drawn from the step's ticket counter, so faster SMs
         // (and the pipelines that got shorter units) take more.
         constexpr int kStatic = 6;
+        const bool alternate = p.hdr->longest_first != 0;
         const uint32_t first_dynamic = static_cast<uint32_t>(kStatic) * 2u * gridDim.x;
         auto draw = [&]() {                              // next unit index (lane 0 draws, all lanes get it)
             uint32_t t = 0;
@@ -376,7 +377,7 @@ hpd_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         };
         auto fixed = [&](int i) {
             const uint32_t j = 2u * blockIdx.x + static_cast<uint32_t>(x);
-            const uint32_t in_round = (i & 1) ? 2u * gridDim.x - 1u - j : j;
+            const uint32_t in_round = ((i & 1) && alternate) ? 2u * gridDim.x - 1u - j : j;
             return static_cast<int>(min(in_round + static_cast<uint32_t>(i) * 2u * gridDim.x, static_cast<uint32_t>(n_units)));
         };
         int w0 = fixed(0), w1 = fixed(1), w2 = fixed(2), w3 = fixed(3);

@@ -58,7 +58,8 @@ struct WsHeader {
     uint32_t ticket;         // dynamic scheduler: next work item
     uint32_t finished;       // CTAs that have drained the list (the last one resets both)
     int32_t work_cap, part_cap;
-    int32_t pad[24];
+    int32_t longest_first;   // 1 if the list is in descending order of the units' estimated duration
+    int32_t pad[23];
 };
 static_assert(sizeof(WsHeader) == 128, "header size");
 

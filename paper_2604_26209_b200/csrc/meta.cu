@@ -424,6 +424,7 @@ __device__ __forceinline__ void plan_block(int n_docs, int G, int Hkv, int n_sm,
         hdr->chunk_tokens = (cand == kCand - 1) ? 0 : (kTileN << cand);
         hdr->n_part_rows = run_part;
         hdr->any_split = split_any;
+        hdr->longest_first = sorted ? 1 : 0;
         hdr->ticket = 0;
         hdr->finished = 0;
         hdr->work_cap = work_cap;
@@ -667,7 +668,7 @@ prefill_meta_kernel(int n_docs, int G, int32_t pos_gap,
         if (threadIdx.x == 0) {
             *n_tokens = n_tok;
             hdr->n_work = n_items; hdr->chunk_tokens = 0; hdr->n_part_rows = 0; hdr->any_split = 0;
-            hdr->ticket = 0; hdr->finished = 0; hdr->work_cap = work_cap; hdr->part_cap = part_cap;
+            hdr->ticket = 0; hdr->finished = 0; hdr->work_cap = work_cap; hdr->part_cap = part_cap; hdr->longest_first = 0;
         }
     }
 }
